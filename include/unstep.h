@@ -1,0 +1,138 @@
+/*
+ * unstep.h -- C ABI of the B200 (sm_100a) chunk-attention library.
+ *
+ * One self-attention layer of a chunk-causal video DiT, for one new latent chunk
+ * (UnStep paper, Sec. "Increasing model efficiency" / "DiT runtime stack" and
+ * appendix "Diffusion transformer runtime", appendix "KV attention window"):
+ *
+ *   1. unstep_rope_table      build the cached float32 cos/sin table of the chunk
+ *   2. unstep_rope_kv_append  rotate Q and K, write K and V into the KV ring
+ *   3. unstep_window_attn     attention of the chunk's queries over the window
+ *
+ * Conventions
+ *   - Every tensor pointer is a DEVICE pointer unless the comment says HOST.
+ *   - bf16 tensors are dense, row-major, 16-byte aligned; the caller owns all of
+ *     them.  The library allocates no device memory.
+ *   - All work is enqueued on `cuda_stream` (a cudaStream_t passed as void*; NULL
+ *     is the legacy default stream).  No call synchronises or reads device data.
+ *   - Return value: 0 on success, a negative unstep_status otherwise.  Arguments
+ *     are validated before anything is launched; on error nothing was enqueued.
+ *   - Chunk positions are plain host integers (the paper keeps the cache
+ *     positions on the CPU so that no call needs a device-to-host read).
+ *
+ * Notation: B streams, Hn heads, D = 128, Fc chunk frames, T = grid_h*grid_w
+ * tokens per latent frame, L = Fc*T queries per chunk, C ring capacity in
+ * frames, token n = (f*grid_h + r)*grid_w + c.
+ */
+#ifndef UNSTEP_H_
+#define UNSTEP_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  UNSTEP_OK = 0,
+  UNSTEP_ERR_INVALID_ARG = -1, /* null or misaligned pointer, bad size, bad window */
+  UNSTEP_ERR_UNSUPPORTED = -2, /* head_dim != 128, device is not sm_100 */
+  UNSTEP_ERR_CUDA = -3,        /* a CUDA runtime/driver call failed */
+  UNSTEP_ERR_TIMEOUT = -4      /* a bounded device-side wait expired (see unstep_poll_status) */
+} unstep_status;
+
+typedef struct {
+  int32_t batch;        /* B: independent streams, each with its own ring */
+  int32_t heads;        /* Hn */
+  int32_t head_dim;     /* D, must be 128 */
+  int32_t chunk_frames; /* Fc: latent frames per chunk */
+  int32_t grid_h;       /* token rows per latent frame */
+  int32_t grid_w;       /* token columns per latent frame; T = grid_h * grid_w */
+  int32_t ring_frames;  /* C: capacity of the KV ring in latent frames */
+  int32_t band_t;       /* head dims rotated by the frame position   (44) */
+  int32_t band_h;       /* head dims rotated by the row position     (42) */
+  int32_t band_w;       /* head dims rotated by the column position  (42) */
+  double rope_base;     /* 10000.0 */
+} unstep_shape_t;
+
+/*
+ * RoPE coefficient table of one chunk (appendix "Diffusion transformer runtime":
+ * float32 sine and cosine tables, one coefficient vector per token, shared by all
+ * heads, built once per starting latent frame index and grid size).
+ *
+ * Pair j in [0, 64) rotates (x[2j], x[2j+1]).  Pairs are split t | h | w in that
+ * order, band_t/2, band_h/2, band_w/2 pairs; local pair i of a band of d_b dims has
+ * omega = rope_base^(-2i/d_b); the angle is position * omega with the position
+ * start_frame + f, r or c; angle and trig are evaluated in double and rounded once.
+ *
+ *   cos_out, sin_out : float32 [L, 64], written.
+ *   start_frame      : absolute latent-frame index of the chunk's first frame, >= 0.
+ * batch, heads and ring_frames of `shape` are not used by this call.
+ */
+int unstep_rope_table(const unstep_shape_t* shape, int32_t start_frame, float* cos_out,
+                      float* sin_out, void* cuda_stream);
+
+/*
+ * Fused RoPE + KV-cache write (Sec. "DiT runtime stack": one kernel loads bf16,
+ * rotates in float32, stores bf16; appendix: newly computed keys and values are
+ * written at the chunk's cache position and repeated denoising calls overwrite the
+ * same entries).
+ *
+ * For every stream b, token n, head h, pair j, with c = cos[n][j], s = sin[n][j]:
+ *     y_even = fl32(fl32(x_even*c) - fl32(x_odd*s))
+ *     y_odd  = fl32(fl32(x_even*s) + fl32(x_odd*c))        (no fused multiply-add)
+ * rounded to bf16 (nearest even).  q_out = rot(q_in); ring_k[b][slot][t] = rot(k_in),
+ * ring_v[b][slot][t] = v_in (bit copy), slot = (start_frame[b] + f) mod C, where
+ * n = f*T + t.  Slots of other frames are not touched.
+ *
+ *   start_frame : HOST int32 [B], each >= 0.
+ *   q_in, k_in, v_in : bf16 [B, L, Hn, 128], read.
+ *   cos, sin    : float32 [L, 64] per table; stream b uses the table at
+ *                 cos + b*table_stream_stride (elements); stride 0 shares one table.
+ *   q_out       : bf16 [B, L, Hn, 128], written; may be the same buffer as q_in.
+ *   ring_k, ring_v : bf16 [B, C, T, Hn, 128], updated in place.
+ */
+int unstep_rope_kv_append(const unstep_shape_t* shape, const int32_t* start_frame,
+                          const void* q_in, const void* k_in, const void* v_in, const float* cos,
+                          const float* sin, int64_t table_stream_stride, void* q_out, void* ring_k,
+                          void* ring_v, void* cuda_stream);
+
+/*
+ * Windowed attention of the chunk's queries (appendix "KV attention window": the
+ * chunk attends the retained most recent latent frames, the current chunk included;
+ * Sec. "DiT runtime stack": fixed-length attention, lengths taken from the call).
+ *
+ * Stream b attends the frames p in [max(0, start_frame[b] + Fc - window_frames),
+ * start_frame[b] + Fc), all T tokens of each, read from ring slot p mod C.  No mask:
+ *     out[b][n][h] = softmax_m( q_rot[b][n][h] . k_m / sqrt(128) ) v_m
+ * bf16 operands, float32 accumulation, bf16 result.
+ *
+ *   start_frame   : HOST int32 [B], each >= 0.
+ *   window_frames : Fc <= window_frames <= C.
+ *   q_rot         : bf16 [B, L, Hn, 128], the q_out of unstep_rope_kv_append.
+ *   ring_k, ring_v: bf16 [B, C, T, Hn, 128], read.  Every attended frame must have
+ *                   been appended and not yet overwritten (true when chunks arrive in
+ *                   order and window_frames <= C).
+ *   out           : bf16 [B, L, Hn, 128], written.
+ */
+int unstep_window_attn(const unstep_shape_t* shape, const int32_t* start_frame,
+                       int32_t window_frames, const void* q_rot, const void* ring_k,
+                       const void* ring_v, void* out, void* cuda_stream);
+
+/* Static, human-readable text for a status code. */
+const char* unstep_strerror(int code);
+
+/*
+ * Device status word of the current device: 0, or UNSTEP_ERR_TIMEOUT if a kernel gave
+ * up on a bounded wait since the last poll (the word is cleared by the poll).  This
+ * call synchronises the device; it is a diagnostic, not part of the hot path.
+ */
+int unstep_poll_status(void);
+
+/* Number of kernels the library has launched in this process (all devices). */
+int64_t unstep_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* UNSTEP_H_ */

@@ -1,0 +1,18 @@
+"""B200 (sm_100a) chunk-attention hot path of a causal video DiT: RoPE table,
+fused RoPE + KV-ring append, windowed attention.  All computation happens in the
+CUDA library behind the C ABI declared in include/unstep.h; this package only
+marshals arguments.  There is no CPU fallback: without the library or a GPU the
+calls raise."""
+
+from .binding import (  # noqa: F401
+    UnstepError,
+    Shape,
+    lib,
+    rope_table,
+    rope_kv_append,
+    window_attn,
+    poll_status,
+    launch_count,
+    strerror,
+    EXPORTS,
+)

@@ -1,0 +1,180 @@
+// RoPE coefficient table and the fused RoPE + KV-ring append (HBM-bound kernels).
+#include <cuda_bf16.h>
+
+#include "common.h"
+
+namespace unstep {
+
+// --------------------------------------------------------------------------
+// Table: one thread per (token, pair).  Angle and trig in double, one rounding.
+// --------------------------------------------------------------------------
+struct TableParams {
+  int32_t start_frame, grid_h, grid_w, L;
+  int32_t pairs_t, pairs_h;  // pairs_w = 64 - pairs_t - pairs_h
+  int32_t band_t, band_h, band_w;
+  double base;
+};
+
+__global__ void __launch_bounds__(256) rope_table_kernel(TableParams p, float* __restrict__ cos_out,
+                                                         float* __restrict__ sin_out) {
+  const int idx = blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= p.L * kPairs) return;
+  const int n = idx >> 6, j = idx & 63;
+  const int T = p.grid_h * p.grid_w;
+  const int f = n / T, t = n - f * T;
+  const int r = t / p.grid_w, c = t - r * p.grid_w;
+  int i, d, pos;
+  if (j < p.pairs_t) {
+    i = j; d = p.band_t; pos = p.start_frame + f;
+  } else if (j < p.pairs_t + p.pairs_h) {
+    i = j - p.pairs_t; d = p.band_h; pos = r;
+  } else {
+    i = j - p.pairs_t - p.pairs_h; d = p.band_w; pos = c;
+  }
+  const double omega = pow(p.base, -(2.0 * static_cast<double>(i)) / static_cast<double>(d));
+  const double theta = static_cast<double>(pos) * omega;
+  double sn, cs;
+  sincos(theta, &sn, &cs);
+  cos_out[idx] = static_cast<float>(cs);
+  sin_out[idx] = static_cast<float>(sn);
+}
+
+// --------------------------------------------------------------------------
+// Append: one thread per 16-byte vector (8 bf16 = 4 pairs) of the same position in
+// q, k and v.  Inputs are read once (streaming loads); outputs are re-read by the
+// attention kernel right after, so they are left to the default cache policy.
+// --------------------------------------------------------------------------
+struct AppendParams {
+  int32_t L, T, C, vec_per_token;  // vec_per_token = Hn * 16
+  int64_t vec_per_stream;          // L * Hn * 16
+  int64_t ring_vec_per_stream;     // C * T * Hn * 16
+  int64_t table_stream_stride;     // elements
+  int32_t slot0[kMaxStreamsPerLaunch];  // start_frame[b] mod C
+};
+
+__device__ __forceinline__ uint32_t rotate_pair(uint32_t w, float c, float s) {
+  const float xe = __uint_as_float(w << 16);
+  const float xo = __uint_as_float(w & 0xFFFF0000u);
+  // four products, one difference, one sum, each rounded to float32: no contraction
+  const float ye = __fsub_rn(__fmul_rn(xe, c), __fmul_rn(xo, s));
+  const float yo = __fadd_rn(__fmul_rn(xe, s), __fmul_rn(xo, c));
+  const __nv_bfloat162 y = __floats2bfloat162_rn(ye, yo);
+  return *reinterpret_cast<const uint32_t*>(&y);
+}
+
+__device__ __forceinline__ uint4 rotate_vec(uint4 x, float4 c, float4 s) {
+  uint4 y;
+  y.x = rotate_pair(x.x, c.x, s.x);
+  y.y = rotate_pair(x.y, c.y, s.y);
+  y.z = rotate_pair(x.z, c.z, s.z);
+  y.w = rotate_pair(x.w, c.w, s.w);
+  return y;
+}
+
+__global__ void __launch_bounds__(256)
+rope_kv_append_kernel(AppendParams p, const uint4* q_in, const uint4* __restrict__ k_in,
+                      const uint4* __restrict__ v_in, const float4* __restrict__ cos_t,
+                      const float4* __restrict__ sin_t, uint4* q_out,
+                      uint4* __restrict__ ring_k, uint4* __restrict__ ring_v) {
+  const int b = blockIdx.y;
+  const int64_t v = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+  if (v >= p.vec_per_stream) return;
+  const int n = static_cast<int>(v / p.vec_per_token);
+  const int rem = static_cast<int>(v - static_cast<int64_t>(n) * p.vec_per_token);
+  const int f = n / p.T, t = n - f * p.T;
+  int slot = p.slot0[b] + f;
+  slot = slot % p.C;
+
+  const int64_t in_idx = static_cast<int64_t>(b) * p.vec_per_stream + v;
+  const uint4 xq = __ldcs(q_in + in_idx);
+  const uint4 xk = __ldcs(k_in + in_idx);
+  const uint4 xv = __ldcs(v_in + in_idx);
+  const int64_t tab = (static_cast<int64_t>(b) * p.table_stream_stride >> 2) +
+                      static_cast<int64_t>(n) * (kPairs / 4) + (rem & 15);
+  const float4 c = __ldg(cos_t + tab);
+  const float4 s = __ldg(sin_t + tab);
+
+  const int64_t ring_idx = static_cast<int64_t>(b) * p.ring_vec_per_stream +
+                           (static_cast<int64_t>(slot) * p.T + t) * p.vec_per_token + rem;
+  q_out[in_idx] = rotate_vec(xq, c, s);
+  ring_k[ring_idx] = rotate_vec(xk, c, s);
+  ring_v[ring_idx] = xv;
+}
+
+}  // namespace unstep
+
+using namespace unstep;
+
+extern "C" int unstep_rope_table(const unstep_shape_t* shape, int32_t start_frame, float* cos_out,
+                                 float* sin_out, void* cuda_stream) {
+  int rc = check_shape(shape, false);
+  if (rc != UNSTEP_OK) return rc;
+  if (start_frame < 0 || cos_out == nullptr || sin_out == nullptr) return UNSTEP_ERR_INVALID_ARG;
+  if (!aligned16(cos_out) || !aligned16(sin_out)) return UNSTEP_ERR_INVALID_ARG;
+  rc = check_device();
+  if (rc != UNSTEP_OK) return rc;
+  TableParams p;
+  p.start_frame = start_frame;
+  p.grid_h = shape->grid_h;
+  p.grid_w = shape->grid_w;
+  p.L = shape->chunk_frames * shape->grid_h * shape->grid_w;
+  p.pairs_t = shape->band_t / 2;
+  p.pairs_h = shape->band_h / 2;
+  p.band_t = shape->band_t;
+  p.band_h = shape->band_h;
+  p.band_w = shape->band_w;
+  p.base = shape->rope_base;
+  const int64_t total = static_cast<int64_t>(p.L) * kPairs;
+  const unsigned blocks = static_cast<unsigned>((total + 255) / 256);
+  rope_table_kernel<<<blocks, 256, 0, static_cast<cudaStream_t>(cuda_stream)>>>(p, cos_out, sin_out);
+  g_launches.fetch_add(1);
+  return cudaGetLastError() == cudaSuccess ? UNSTEP_OK : UNSTEP_ERR_CUDA;
+}
+
+extern "C" int unstep_rope_kv_append(const unstep_shape_t* shape, const int32_t* start_frame,
+                                     const void* q_in, const void* k_in, const void* v_in,
+                                     const float* cos, const float* sin,
+                                     int64_t table_stream_stride, void* q_out, void* ring_k,
+                                     void* ring_v, void* cuda_stream) {
+  int rc = check_shape(shape, true);
+  if (rc != UNSTEP_OK) return rc;
+  const void* ptrs[] = {start_frame, q_in, k_in, v_in, cos, sin, q_out, ring_k, ring_v};
+  for (const void* ptr : ptrs)
+    if (ptr == nullptr) return UNSTEP_ERR_INVALID_ARG;
+  const void* dev_ptrs[] = {q_in, k_in, v_in, cos, sin, q_out, ring_k, ring_v};
+  for (const void* ptr : dev_ptrs)
+    if (!aligned16(ptr)) return UNSTEP_ERR_INVALID_ARG;
+  if (table_stream_stride < 0 || (table_stream_stride & 3)) return UNSTEP_ERR_INVALID_ARG;
+  for (int b = 0; b < shape->batch; ++b)
+    if (start_frame[b] < 0) return UNSTEP_ERR_INVALID_ARG;
+  rc = check_device();
+  if (rc != UNSTEP_OK) return rc;
+
+  const int64_t T = static_cast<int64_t>(shape->grid_h) * shape->grid_w;
+  const int64_t L = T * shape->chunk_frames;
+  AppendParams p;
+  p.L = static_cast<int32_t>(L);
+  p.T = static_cast<int32_t>(T);
+  p.C = shape->ring_frames;
+  p.vec_per_token = shape->heads * 16;
+  p.vec_per_stream = L * p.vec_per_token;
+  p.ring_vec_per_stream = static_cast<int64_t>(shape->ring_frames) * T * p.vec_per_token;
+  p.table_stream_stride = table_stream_stride;
+  const unsigned blocks = static_cast<unsigned>((p.vec_per_stream + 255) / 256);
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  for (int b0 = 0; b0 < shape->batch; b0 += kMaxStreamsPerLaunch) {
+    const int nb = shape->batch - b0 < kMaxStreamsPerLaunch ? shape->batch - b0 : kMaxStreamsPerLaunch;
+    for (int i = 0; i < nb; ++i) p.slot0[i] = start_frame[b0 + i] % shape->ring_frames;
+    const int64_t in_off = static_cast<int64_t>(b0) * p.vec_per_stream;
+    const int64_t ring_off = static_cast<int64_t>(b0) * p.ring_vec_per_stream;
+    const int64_t tab_off = static_cast<int64_t>(b0) * table_stream_stride;
+    rope_kv_append_kernel<<<dim3(blocks, nb), 256, 0, st>>>(
+        p, static_cast<const uint4*>(q_in) + in_off, static_cast<const uint4*>(k_in) + in_off,
+        static_cast<const uint4*>(v_in) + in_off, reinterpret_cast<const float4*>(cos + tab_off),
+        reinterpret_cast<const float4*>(sin + tab_off), static_cast<uint4*>(q_out) + in_off,
+        static_cast<uint4*>(ring_k) + ring_off, static_cast<uint4*>(ring_v) + ring_off);
+    g_launches.fetch_add(1);
+    if (cudaGetLastError() != cudaSuccess) return UNSTEP_ERR_CUDA;
+  }
+  return UNSTEP_OK;
+}
