@@ -113,7 +113,8 @@ def rope_angles(start_frame, chunk_frames, grid_h, grid_w, bands=(44, 42, 42), b
 def rope_table(start_frame, chunk_frames, grid_h, grid_w, bands=(44, 42, 42), base=10000.0):
     """The cached table of R2: (cos, sin), float32 [L, 64], one rounding from fp64."""
     theta = rope_angles(start_frame, chunk_frames, grid_h, grid_w, bands, base)
-    return np.cos(theta).astype(np.float32), np.sin(theta).astype(np.float32)
+    return (np.ascontiguousarray(np.cos(theta), dtype=np.float32),
+            np.ascontiguousarray(np.sin(theta), dtype=np.float32))
 
 
 # ---------------------------------------------------------------------------
