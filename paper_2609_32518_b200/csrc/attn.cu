@@ -1,10 +1,19 @@
-// Windowed attention of one chunk over the KV ring: TMA-staged tiles, tcgen05 MMA
-// into TMEM for Q K^T and P V, online softmax in registers.
+// Windowed attention of one chunk over the KV ring (sm_100a).
 //
-// Work item = (stream b, head h, 128-query tile).  Keys are walked frame by frame:
-// frame p of the window lives in ring slot p mod C, and every 128-key tile lies
-// inside one frame, so the 5-D tensor map (d, head, token, slot, stream) zero-fills
-// the ragged end of a frame and the ring never has to be copied or linearised.
+// Persistent, warp-specialised kernel, one CTA per SM:
+//   warps 0-3   softmax of query tile 0 (one thread per query row)
+//   warps 4-7   softmax of query tile 1
+//   warp  8, 9  tcgen05.mma issuers of query tile 0 and 1 (one lane each); warp 8 owns TMEM
+//   warp  10    TMA producer (one lane)
+// A work item is (stream, head, pair of 128-query tiles): both tiles share every K/V
+// tile, and the softmax of one overlaps the tensor-core work of the other.  S = Q K^T
+// and O += P V accumulate in TMEM; P (bf16) is written back over S and fed to the
+// second MMA straight from TMEM.
+//
+// Keys are walked frame by frame: frame p of the window lives in ring slot p mod C and
+// every key tile lies inside one frame, so the 5-D tensor map (d, head, token, slot,
+// stream) zero-fills the ragged end of a frame and the ring is never copied.  The last
+// tile of a frame runs with a narrower MMA (N rounded up to 16).
 #include <cuda.h>
 #include <cuda_bf16.h>
 
@@ -19,81 +28,243 @@ using namespace ptx;
 
 __device__ int g_status = 0;
 
-constexpr int kTileM = 128;          // queries per work item
-constexpr int kTileN = 128;          // keys per tile
-constexpr int kHalfBytes = 128 * 64 * 2;   // one TMA box: 128 rows x 64 bf16 (128-byte rows)
-constexpr int kTileBytes = 2 * kHalfBytes; // 128 x 128 bf16
-constexpr int kTmemCols = 256;       // S/P: columns [0,128), O: columns [128,256)
+// Optional timeline of CTA 0 (debug builds only): clock64 stamps per role, tile and event.
+#ifdef UNSTEP_TRACE
+__device__ long long g_trace[4][64][8];
+#define TRACE(role, tile, ev)                                                          \
+  do {                                                                                 \
+    if (blockIdx.x == 0 && (tile) < 64 && (threadIdx.x & 31) == 0 && ((threadIdx.x >> 5) & 3) < 2 && (threadIdx.x < 128 ? threadIdx.x == 0 : true) && (threadIdx.x >= 256 || (threadIdx.x & 127) == 0)) g_trace[role][tile][ev] = clock64(); \
+  } while (0)
+#else
+#define TRACE(role, tile, ev) \
+  do {                        \
+  } while (0)
+#endif
+
+constexpr int kTileM = 128;                 // queries per tile (two tiles per work item)
+constexpr int kTileN = 128;                 // keys per tile
+constexpr int kHalfBytes = 128 * 64 * 2;    // one TMA box: 128 rows x 64 bf16 (128-byte rows)
+constexpr int kTileBytes = 2 * kHalfBytes;  // 128 x 128 bf16
+constexpr int kStages = 5;                  // 32 KB buffers shared by the K and V tiles
+constexpr int kThreads = 384;
+constexpr int kTmemCols = 512;              // S0 | S1 | O0 | O1, 128 fp32 columns each
 constexpr long long kWaitCycles = 2000000000LL;  // about a second: then give up, never hang
+constexpr float kRescaleThreshold = 8.f;    // log2 units: rescale O only when the max grows by 2^8
+
+constexpr int kSmemQ = 0;
+constexpr int kSmemKV = 2 * kTileBytes;
+constexpr int kSmemBar = kSmemKV + kStages * kTileBytes;
+constexpr int kAttnSmemBytes = kSmemBar + 256 + 1024;  // + barriers/flags + alignment slack
 
 struct AttnParams {
   int32_t Hn, L, T, C;
-  int32_t q_tiles;         // ceil(L / 128)
-  int32_t tiles_per_frame; // ceil(T / 128)
-  float scale_log2e;       // log2(e) / sqrt(128)
+  int32_t q_tiles;          // ceil(L / 128)
+  int32_t q_pairs;          // ceil(q_tiles / 2)
+  int32_t tiles_per_frame;  // ceil(T / 128)
+  int32_t tail_valid;       // valid keys in the last tile of a frame, 1..128
+  int32_t n_streams;
+  float scale_log2e;        // log2(e) / sqrt(128)
   int32_t first_frame[kMaxStreamsPerLaunch];  // first attended absolute frame of stream b
   int32_t n_frames[kMaxStreamsPerLaunch];     // attended frames of stream b
 };
 
+// One unit of work of a CTA: key tiles [t0, t1) of item (b, h, query-tile pair qp).
+struct Seg {
+  int b, h, qp, nq, t0, t1;
+};
+
+// Contiguous, balanced split of the items over the CTAs.  Items are ordered stream, head,
+// query pair, so CTAs that run side by side read the same head's K/V through L2.
+struct Sched {
+  int cur, end;
+  const AttnParams& p;
+  __device__ Sched(const AttnParams& prm) : p(prm) {
+    const long long items = static_cast<long long>(p.n_streams) * p.Hn * p.q_pairs;
+    cur = static_cast<int>(items * blockIdx.x / gridDim.x);
+    end = static_cast<int>(items * (blockIdx.x + 1) / gridDim.x);
+  }
+  __device__ bool next(Seg& s) {
+    if (cur >= end) return false;
+    int it = cur++;
+    s.qp = it % p.q_pairs;
+    it /= p.q_pairs;
+    s.h = it % p.Hn;
+    s.b = it / p.Hn;
+    s.nq = (2 * s.qp + 1 < p.q_tiles) ? 2 : 1;
+    s.t0 = 0;
+    s.t1 = p.n_frames[s.b] * p.tiles_per_frame;
+    return true;
+  }
+};
+
 struct Waiter {
   volatile int* abort_flag;
+  // Bounded wait: the hardware parks the thread between polls; the clock and the CTA's abort
+  // flag are only looked at every 32 polls so that a waiting warp leaves the issue slots alone.
   __device__ __forceinline__ bool wait(uint32_t bar, uint32_t parity) const {
     if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
-    while (true) {
-      if (mbar_try_wait(bar, parity)) return true;
-      if (*abort_flag) return false;
-      if (clock64() - t0 > kWaitCycles) {
-        *abort_flag = 1;
-        atomicExch(&g_status, UNSTEP_ERR_TIMEOUT);
-        return false;
+    for (uint32_t spin = 1;; ++spin) {
+      if (mbar_try_wait_hint(bar, parity, 2000u)) return true;
+      if ((spin & 31u) == 0u) {
+        if (*abort_flag) return false;
+        if (clock64() - t0 > kWaitCycles) {
+          *abort_flag = 1;
+          atomicExch(&g_status, UNSTEP_ERR_TIMEOUT);
+          return false;
+        }
       }
     }
   }
 };
 
-__global__ void __launch_bounds__(128, 2)
+__device__ __forceinline__ void reg_dealloc_96() { asm volatile("setmaxnreg.dec.sync.aligned.u32 96;"); }
+__device__ __forceinline__ void reg_alloc_200() { asm volatile("setmaxnreg.inc.sync.aligned.u32 200;"); }
+
+// --------------------------------------------------------------------------------------
+// Softmax of one 128 x 128 score tile for this thread's row.
+//   t_S / t_O  : TMEM addresses (this warp's lanes) of the score and output tiles
+//   kMasked    : columns >= nvalid are excluded (last tile of a frame)
+// The running maximum is only raised when it grows by more than 2^kRescaleThreshold, so
+// the output accumulator is rescaled rarely; P stays below 2^8 in between.  The caller has
+// seen S of this tile complete, which (the tensor pipe runs in issue order) also means the
+// previous P V into O has landed, so O may be rescaled here without another wait.
+// P is handed to the MMA warp in two halves of 64 keys (bar_p_half, bar_p_half + 8).
+// The two warpgroups take turns on the exponentials (bar_turn_wait / bar_turn_signal, 0 = no
+// partner): the MUFU pipe is shared, and alternating keeps the two query tiles half a period
+// apart, so that the tensor pipe always has one tile's MMAs to run while the other tile is
+// in its softmax.  Returns false when a bounded wait gave up.
+// --------------------------------------------------------------------------------------
+template <bool kMasked>
+__device__ __forceinline__ bool softmax_tile(uint32_t t_S, uint32_t t_O, float c, int nvalid,
+                                             bool first, float& m_run, float& l_run,
+                                             uint32_t bar_p_half, const Waiter& w,
+                                             uint32_t bar_turn_wait, uint32_t turn_parity,
+                                             uint32_t bar_turn_signal, int trace_role,
+                                             int trace_tile) {
+  uint32_t sreg[128];
+#pragma unroll
+  for (int q = 0; q < 4; ++q) tmem_ld32(t_S + q * 32, sreg + q * 32);
+  tc_wait_ld();
+  TRACE(trace_role, trace_tile, 2);
+  if (kMasked) {
+#pragma unroll
+    for (int i = 0; i < 128; ++i)
+      if (i >= nvalid) sreg[i] = 0xFF800000u;  // -inf
+  }
+  // row maximum: four independent chains of 3-input max
+  float mx4[4];
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+    float m = fmaxf(__uint_as_float(sreg[32 * q]), __uint_as_float(sreg[32 * q + 1]));
+#pragma unroll
+    for (int i = 2; i < 32; i += 2)
+      m = max3(m, __uint_as_float(sreg[32 * q + i]), __uint_as_float(sreg[32 * q + i + 1]));
+    mx4[q] = m;
+  }
+  const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
+  TRACE(trace_role, trace_tile, 3);
+  float alpha = 1.f;
+  bool grow = false;
+  if (first) {
+    m_run = mx;
+  } else if ((mx - m_run) * c > kRescaleThreshold) {
+    alpha = ex2((m_run - mx) * c);
+    m_run = mx;
+    l_run *= alpha;
+    grow = true;
+  }
+  if (__any_sync(0xFFFFFFFFu, grow)) {
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      uint32_t o[32];
+      tmem_ld32(t_O + q * 32, o);
+      tc_wait_ld();
+#pragma unroll
+      for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
+      tmem_st32(t_O + q * 32, o);
+    }
+  }
+  if (bar_turn_wait != 0u && !w.wait(bar_turn_wait, turn_parity)) return false;
+  TRACE(trace_role, trace_tile, 6);
+  // p = 2^(s*c - m*c): packed FMA on pairs, one MUFU per element, packed partial sums
+  const uint64_t c2 = pack_f32x2(c, c);
+  const float neg_ms = -m_run * c;
+  const uint64_t nm2 = pack_f32x2(neg_ms, neg_ms);
+  uint64_t acc[4] = {0ull, 0ull, 0ull, 0ull};
+#pragma unroll
+  for (int half = 0; half < 2; ++half) {
+    uint32_t preg[32];
+#pragma unroll
+    for (int i = 0; i < 32; ++i) {
+      const uint64_t x2 = fma_f32x2(pack_f32x2(__uint_as_float(sreg[64 * half + 2 * i]),
+                                               __uint_as_float(sreg[64 * half + 2 * i + 1])), c2, nm2);
+      float x0, x1;
+      unpack_f32x2(x2, x0, x1);
+      const float p0 = ex2(x0), p1 = ex2(x1);
+      acc[i & 3] = add_f32x2(acc[i & 3], pack_f32x2(p0, p1));
+      preg[i] = pack_bf16x2(p0, p1);
+    }
+    tmem_st32(t_S + 32 * half, preg);  // P (bf16 pairs) overwrites the first 64 columns of S
+    if (half == 1 && bar_turn_signal != 0u) mbar_arrive(bar_turn_signal);
+    tc_wait_st();
+    tc_fence_before();
+    mbar_arrive(bar_p_half + 8 * half);
+    TRACE(trace_role, trace_tile, 4 + half);
+  }
+  {
+    const uint64_t t = add_f32x2(add_f32x2(acc[0], acc[1]), add_f32x2(acc[2], acc[3]));
+    float t0, t1;
+    unpack_f32x2(t, t0, t1);
+    l_run += t0 + t1;
+  }
+  return true;
+}
+
+__global__ void __launch_bounds__(kThreads, 1)
 window_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                    const __grid_constant__ CUtensorMap tm_v, const AttnParams p,
                    __nv_bfloat16* __restrict__ out) {
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-  const uint32_t sQ = smem_base;
-  const uint32_t sK = sQ + kTileBytes;
-  const uint32_t sV = sK + kTileBytes;
-  const uint32_t sBar = sV + kTileBytes;
-  const uint32_t bar_q = sBar + 0, bar_k = sBar + 8, bar_v = sBar + 16, bar_s = sBar + 24,
-                 bar_o = sBar + 32;
-  uint8_t* gen = smem_raw + (smem_base - smem_u32(smem_raw)) + 3 * kTileBytes;
-  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(gen + 64);
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(gen + 72);
+  uint8_t* gen = smem_raw + (smem_base - smem_u32(smem_raw));
+  const uint32_t sQ = smem_base + kSmemQ;
+  const uint32_t sKV = smem_base + kSmemKV;
+  const uint32_t sBar = smem_base + kSmemBar;
+  // mbarriers (8 bytes each)
+  const uint32_t bar_q_full = sBar;                          // [2]  TMA -> MMA warp a
+  const uint32_t bar_q_empty = sBar + 16;                    // [2]  MMA warp a -> TMA
+  const uint32_t bar_kv_full = sBar + 32;                    // [kStages] TMA -> both MMA warps
+  const uint32_t bar_kv_empty = sBar + 32 + 8 * kStages;     // [kStages] both MMA warps -> TMA
+  const uint32_t bar_s_full = sBar + 32 + 16 * kStages;      // [2]  MMA warp a -> softmax a
+  const uint32_t bar_p_half = bar_s_full + 16;               // [2][2] softmax a -> MMA warp a
+  const uint32_t bar_o_final = bar_p_half + 32;              // [2]  MMA warp a -> softmax a
+  const uint32_t bar_turn = bar_o_final + 16;                // [2]  softmax 1-a -> softmax a
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(gen + kSmemBar + 192);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(gen + kSmemBar + 200);
 
   const int tid = threadIdx.x;
   const int warp = tid >> 5;
-
-  // work item: q tile fastest, then head, then stream, so neighbouring CTAs share K/V in L2
-  int item = blockIdx.x;
-  const int qt = item % p.q_tiles;
-  item /= p.q_tiles;
-  const int h = item % p.Hn;
-  const int b = item / p.Hn;
-  const int n0 = qt * kTileM;
-  const int first_frame = p.first_frame[b];
-  const int total_tiles = p.n_frames[b] * p.tiles_per_frame;
+  const int lane = tid & 31;
 
   if (tid == 0) {
-    mbar_init(bar_q, 1);
-    mbar_init(bar_k, 1);
-    mbar_init(bar_v, 1);
-    mbar_init(bar_s, 1);
-    mbar_init(bar_o, 1);
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(bar_q_full + 8 * i, 1);
+      mbar_init(bar_q_empty + 8 * i, 1);
+      mbar_init(bar_s_full + 8 * i, 1);
+      mbar_init(bar_p_half + 16 * i, 128);
+      mbar_init(bar_p_half + 16 * i + 8, 128);
+      mbar_init(bar_o_final + 8 * i, 1);
+      mbar_init(bar_turn + 8 * i, 128);
+    }
+    for (int i = 0; i < kStages; ++i) {
+      mbar_init(bar_kv_full + 8 * i, 1);
+      mbar_init(bar_kv_empty + 8 * i, 2);
+    }
     *abort_flag = 0;
     mbar_fence_init();
-    prefetch_tensormap(&tm_q);
-    prefetch_tensormap(&tm_k);
-    prefetch_tensormap(&tm_v);
   }
-  if (warp == 0) {
+  if (warp == 8) {
     tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), kTmemCols);
     tmem_relinquish();
   }
@@ -101,173 +272,241 @@ window_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
-  const uint32_t t_lane = tmem_base + (static_cast<uint32_t>(warp * 32) << 16);
-  const uint32_t t_S = t_lane;        // this warp's 32 lanes, columns [0, 128)
-  const uint32_t t_O = t_lane + 128;  // columns [128, 256)
   const Waiter w{abort_flag};
+  const int tail_n = (p.tail_valid + 15) & ~15;  // MMA N of the last tile of a frame
 
-  constexpr uint32_t kIdescQK = idesc_bf16_f32(kTileM, kTileN, 0);
-  constexpr uint32_t kIdescPV = idesc_bf16_f32(kTileM, kHeadDim, 1);
-
-  auto issue_kv_load = [&](uint32_t dst, const CUtensorMap* tm, uint32_t bar, int j) {
-    const int fi = j / p.tiles_per_frame;
-    const int tok0 = (j - fi * p.tiles_per_frame) * kTileN;
-    const int slot = (first_frame + fi) % p.C;
-    mbar_expect_tx(bar, kTileBytes);
-    tma_load_5d(dst, tm, bar, 0, h, tok0, slot, b);
-    tma_load_5d(dst + kHalfBytes, tm, bar, 64, h, tok0, slot, b);
-  };
-
-  bool k_inflight = false, v_inflight = false, q_inflight = false;
-  if (tid == 0) {
-    mbar_expect_tx(bar_q, kTileBytes);
-    tma_load_4d(sQ, &tm_q, bar_q, 0, h, n0, b);
-    tma_load_4d(sQ + kHalfBytes, &tm_q, bar_q, 64, h, n0, b);
-    issue_kv_load(sK, &tm_k, bar_k, 0);
-    issue_kv_load(sV, &tm_v, bar_v, 0);
-    q_inflight = k_inflight = v_inflight = true;
-  }
-
-  float m_run = -INFINITY, l_run = 0.f;
-  bool ok = true;
-
-  for (int j = 0; j < total_tiles && ok; ++j) {
-    const uint32_t ph = j & 1;
-    const int fi = j / p.tiles_per_frame;
-    const int tok0 = (j - fi * p.tiles_per_frame) * kTileN;
-    const int nvalid = min(kTileN, p.T - tok0);
-
-    // ---- S = Q K^T -------------------------------------------------------
-    if (tid == 0) {
-      if (j == 0) {
-        ok = w.wait(bar_q, 0);
-        q_inflight = false;
+  if (warp >= 8) {
+    reg_dealloc_96();
+    if (warp == 10 && lane == 0) {
+      // ------------------------------------------------------------ TMA producer
+      prefetch_tensormap(&tm_q);
+      prefetch_tensormap(&tm_k);
+      prefetch_tensormap(&tm_v);
+      Sched sched(p);
+      Seg s;
+      uint32_t kv_it = 0, q_it[2] = {0, 0};
+      bool ok = true;
+      while (ok && sched.next(s)) {
+        for (int a = 0; a < s.nq && ok; ++a) {
+          ok = w.wait(bar_q_empty + 8 * a, (q_it[a] & 1) ^ 1);
+          if (!ok) break;
+          const uint32_t dst = sQ + a * kTileBytes, bar = bar_q_full + 8 * a;
+          const int n0 = (2 * s.qp + a) * kTileM;
+          mbar_expect_tx(bar, kTileBytes);
+          tma_load_4d(dst, &tm_q, bar, 0, s.h, n0, s.b);
+          tma_load_4d(dst + kHalfBytes, &tm_q, bar, 64, s.h, n0, s.b);
+          ++q_it[a];
+        }
+        const int first_frame = p.first_frame[s.b];
+        int fi = s.t0 / p.tiles_per_frame;
+        int ti = s.t0 - fi * p.tiles_per_frame;
+        for (int j = s.t0; j < s.t1 && ok; ++j) {
+          const int slot_f = (first_frame + fi) % p.C;
+          const int tok0 = ti * kTileN;
+          for (int kv = 0; kv < 2 && ok; ++kv) {
+            const uint32_t st = kv_it % kStages;
+            ok = w.wait(bar_kv_empty + 8 * st, ((kv_it / kStages) & 1) ^ 1);
+            if (!ok) break;
+            const uint32_t dst = sKV + st * kTileBytes, bar = bar_kv_full + 8 * st;
+            const CUtensorMap* tm = kv == 0 ? &tm_k : &tm_v;
+            mbar_expect_tx(bar, kTileBytes);
+            tma_load_5d(dst, tm, bar, 0, s.h, tok0, slot_f, s.b);
+            tma_load_5d(dst + kHalfBytes, tm, bar, 64, s.h, tok0, slot_f, s.b);
+            ++kv_it;
+          }
+          if (++ti == p.tiles_per_frame) {
+            ti = 0;
+            ++fi;
+          }
+        }
       }
-      if (ok) ok = w.wait(bar_k, ph);
-      if (ok) {
-        k_inflight = false;
+    } else if (warp <= 9 && lane == 0) {
+      // ------------------------------------------------------------ MMA issuer of query tile a
+      // One issuing thread per query tile, on different scheduler partitions.  For each key
+      // tile: O_a += P_a V (two halves, as P arrives), then S_a = Q_a K_next^T.  Both warps
+      // walk the same K/V ring; a stage is released when both have retired it.
+      const int a = warp - 8;
+      Sched sched(p);
+      Seg s;
+      uint32_t kv_it = 0, q_it = 0, sp_it = 0;
+      bool ok = true;
+      const uint32_t idesc_pv = idesc_bf16_f32(kTileM, kHeadDim, 1);
+      const uint32_t idesc_qk_full = idesc_bf16_f32(kTileM, kTileN, 0);
+      const uint32_t idesc_qk_tail = idesc_bf16_f32(kTileM, tail_n, 0);
+      const int k_steps_tail = tail_n >> 4;
+      // descriptors are built once; per instruction only the start-address field moves
+      const uint64_t dq = smem_desc_sw128(sQ + a * kTileBytes, 16, 1024);   // Q tile a, K-major
+      const uint64_t dk0 = smem_desc_sw128(sKV, 16, 1024);                  // stage 0 as a K tile
+      const uint64_t dv0 = smem_desc_sw128(sKV, kHalfBytes, 1024);          // stage 0 as a V tile (MN-major)
+      const uint32_t s_tmem = tmem_base + a * 128, o_tmem = tmem_base + 256 + a * 128;
+      const uint32_t my_s_full = bar_s_full + 8 * a, my_p_half = bar_p_half + 16 * a;
+
+      auto issue_qk = [&](uint32_t stage, bool tail) {
+        const uint64_t dk = dk0 + static_cast<uint64_t>((stage * kTileBytes) >> 4);
+        const uint32_t idesc = tail ? idesc_qk_tail : idesc_qk_full;
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+          const uint64_t off = static_cast<uint64_t>(((k >> 2) * kHalfBytes + (k & 3) * 32) >> 4);
+          mma_ss(s_tmem, dq + off, dk + off, idesc, k > 0);
+        }
+        tc_commit(my_s_full);
+        tc_commit(bar_kv_empty + 8 * stage);
+      };
+      auto issue_pv_half = [&](uint64_t dv, int half, int k_steps, bool accumulate) {
+#pragma unroll
+        for (int k = 4 * half; k < 4 * half + 4; ++k)
+          if (k < k_steps)
+            mma_ts(o_tmem, s_tmem + k * 8, dv + static_cast<uint64_t>((k * 2048) >> 4), idesc_pv,
+                   (accumulate || k > 0) ? 1u : 0u);
+      };
+
+      while (ok && sched.next(s)) {
+        const bool part = a < s.nq;   // a lone last query tile leaves warp 1 only the bookkeeping
+        const int n = s.t1 - s.t0;
+        int ti = s.t0 % p.tiles_per_frame;  // tile index inside its frame
+        if (part) {
+          ok = w.wait(bar_q_full + 8 * a, q_it & 1);
+          if (!ok) break;
+          ++q_it;
+        }
+        uint32_t kst = kv_it % kStages;
+        ok = w.wait(bar_kv_full + 8 * kst, (kv_it / kStages) & 1);
+        if (!ok) break;
+        ++kv_it;
+        if (part) {
+          tc_fence_after();
+          issue_qk(kst, ti == p.tiles_per_frame - 1);
+        } else {
+          mbar_arrive(bar_kv_empty + 8 * kst);
+        }
+        for (int j = 0; j < n; ++j) {
+          const int k_steps = (ti == p.tiles_per_frame - 1) ? k_steps_tail : 8;
+          if (++ti == p.tiles_per_frame) ti = 0;
+          const uint32_t vst = kv_it % kStages;
+          ok = w.wait(bar_kv_full + 8 * vst, (kv_it / kStages) & 1);
+          if (!ok) break;
+          ++kv_it;
+          const bool more = j + 1 < n;
+          if (more) {
+            kst = kv_it % kStages;
+            ok = w.wait(bar_kv_full + 8 * kst, (kv_it / kStages) & 1);
+            if (!ok) break;
+            ++kv_it;
+          }
+          if (part) {
+            const uint64_t dv = dv0 + static_cast<uint64_t>((vst * kTileBytes) >> 4);
+            TRACE(2 + a, sp_it, 0);
+            ok = w.wait(my_p_half, sp_it & 1);
+            if (!ok) break;
+            TRACE(2 + a, sp_it, 1);
+            tc_fence_after();
+            issue_pv_half(dv, 0, k_steps, j > 0);
+            TRACE(2 + a, sp_it, 2);
+            ok = w.wait(my_p_half + 8, sp_it & 1);
+            if (!ok) break;
+            TRACE(2 + a, sp_it, 3);
+            tc_fence_after();
+            issue_pv_half(dv, 1, k_steps, true);
+            tc_commit(bar_kv_empty + 8 * vst);
+            TRACE(2 + a, sp_it, 4);
+            if (more) issue_qk(kst, ti == p.tiles_per_frame - 1);
+            TRACE(2 + a, sp_it, 5);
+            ++sp_it;
+          } else {
+            mbar_arrive(bar_kv_empty + 8 * vst);
+            if (more) mbar_arrive(bar_kv_empty + 8 * kst);
+          }
+        }
+        if (!ok) break;
+        if (part) {
+          tc_commit(bar_o_final + 8 * a);
+          tc_commit(bar_q_empty + 8 * a);
+        }
+      }
+    }
+  } else {
+    // ---------------------------------------------------------------- softmax warpgroups
+    reg_alloc_200();
+    const int a = warp >> 2;               // query tile of this warpgroup
+    const int row = tid & 127;             // row inside the tile = TMEM lane
+    const uint32_t t_lane = tmem_base + (static_cast<uint32_t>((warp & 3) * 32) << 16);
+    const uint32_t t_S = t_lane + a * 128;
+    const uint32_t t_O = t_lane + 256 + a * 128;
+    const uint32_t my_s_full = bar_s_full + 8 * a, my_p_half = bar_p_half + 16 * a,
+                   my_o_final = bar_o_final + 8 * a;
+    Sched sched(p);
+    Seg s;
+    uint32_t it = 0, seg_it = 0, pair_it = 0;  // pair_it: tiles seen while both warpgroups work
+    bool ok = true;
+    while (ok && sched.next(s)) {
+      if (a >= s.nq) continue;
+      const bool paired = s.nq == 2;
+      const uint32_t turn_wait = paired ? bar_turn + 8 * a : 0u;
+      const uint32_t turn_signal = paired ? bar_turn + 8 * (1 - a) : 0u;
+      float m_run = -INFINITY, l_run = 0.f;
+      int ti = s.t0 % p.tiles_per_frame;
+      for (int j = s.t0; j < s.t1; ++j) {
+        TRACE(a, it, 0);
+        ok = w.wait(my_s_full, it & 1);
+        if (!ok) break;
         tc_fence_after();
-#pragma unroll
-        for (int k = 0; k < 8; ++k) {
-          const uint32_t off = (k >> 2) * kHalfBytes + (k & 3) * 32;
-          mma_ss(tmem_base, smem_desc_sw128(sQ + off, 16, 1024), smem_desc_sw128(sK + off, 16, 1024),
-                 kIdescQK, k > 0);
-        }
-        tc_commit(bar_s);
+        TRACE(a, it, 1);
+        const bool tail = (ti == p.tiles_per_frame - 1);
+        if (++ti == p.tiles_per_frame) ti = 0;
+        // tile 0 waits for tile 1's previous tile, tile 1 for tile 0's current one
+        const uint32_t turn_parity = (a == 0) ? ((pair_it & 1) ^ 1) : (pair_it & 1);
+        if (tail && p.tail_valid < kTileN)
+          ok = softmax_tile<true>(t_S, t_O, p.scale_log2e, p.tail_valid, j == s.t0, m_run, l_run, my_p_half,
+                                  w, turn_wait, turn_parity, turn_signal, a, it);
+        else
+          ok = softmax_tile<false>(t_S, t_O, p.scale_log2e, kTileN, j == s.t0, m_run, l_run, my_p_half,
+                                   w, turn_wait, turn_parity, turn_signal, a, it);
+        if (!ok) break;
+        ++it;
+        if (paired) ++pair_it;
       }
-    }
-    if (!w.wait(bar_s, ph)) { ok = false; break; }
-    tc_fence_after();
-    if (tid == 0 && j + 1 < total_tiles) {  // K tile is consumed: prefetch the next one
-      issue_kv_load(sK, &tm_k, bar_k, j + 1);
-      k_inflight = true;
-    }
-
-    // ---- online softmax on this thread's row ----------------------------
-    uint32_t sreg[128];
-#pragma unroll
-    for (int c = 0; c < 4; ++c) tmem_ld32(t_S + c * 32, sreg + c * 32);
-    tc_wait_ld();
-    float mx = -INFINITY;
-#pragma unroll
-    for (int i = 0; i < 128; ++i) {
-      float s = __uint_as_float(sreg[i]);
-      if (i >= nvalid) s = -INFINITY;
-      sreg[i] = __float_as_uint(s);
-      mx = fmaxf(mx, s);
-    }
-    const float m_new = fmaxf(m_run, mx);
-    const float alpha = ex2((m_run - m_new) * p.scale_log2e);
-    const float neg_ms = -m_new * p.scale_log2e;
-    float psum = 0.f;
-    // P (bf16, two per column) overwrites the first 64 columns of S, 32 columns at a time
-#pragma unroll
-    for (int half = 0; half < 2; ++half) {
-      uint32_t preg[32];
-#pragma unroll
-      for (int i = 0; i < 32; ++i) {
-        const float p0 = ex2(fmaf(__uint_as_float(sreg[64 * half + 2 * i]), p.scale_log2e, neg_ms));
-        const float p1 = ex2(fmaf(__uint_as_float(sreg[64 * half + 2 * i + 1]), p.scale_log2e, neg_ms));
-        psum += p0 + p1;
-        preg[i] = pack_bf16x2(p0, p1);
-      }
-      tmem_st32(t_S + 32 * half, preg);
-    }
-    l_run = fmaf(l_run, alpha, psum);
-    m_run = m_new;
-    // rescale the running output when some row of the warp moved its maximum
-    if (j > 0 && __any_sync(0xFFFFFFFFu, alpha != 1.f)) {
-#pragma unroll
-      for (int c = 0; c < 4; ++c) {
-        uint32_t o[32];
-        tmem_ld32(t_O + c * 32, o);
-        tc_wait_ld();
-#pragma unroll
-        for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
-        tmem_st32(t_O + c * 32, o);
-      }
-    }
-    tc_wait_st();
-    tc_fence_before();
-    __syncthreads();
-
-    // ---- O += P V ---------------------------------------------------------
-    if (tid == 0) {
+      if (!ok) break;
+      // epilogue: wait for the last P V, then O / l -> bf16 -> out[b][n][h][:]
+      ok = w.wait(my_o_final, seg_it & 1);
+      if (!ok) break;
+      ++seg_it;
       tc_fence_after();
-      ok = w.wait(bar_v, ph);
-      if (ok) {
-        v_inflight = false;
+      const int n = (2 * s.qp + a) * kTileM + row;
+      const float inv_l = 1.f / l_run;
+      uint4* dst = reinterpret_cast<uint4*>(
+          out + ((static_cast<int64_t>(s.b) * p.L + n) * p.Hn + s.h) * kHeadDim);
 #pragma unroll
-        for (int k = 0; k < 8; ++k) {
-          mma_ts(tmem_base + 128, tmem_base + k * 8, smem_desc_sw128(sV + k * 2048, kHalfBytes, 1024),
-                 kIdescPV, (j > 0 || k > 0) ? 1u : 0u);
+      for (int q = 0; q < 4; ++q) {
+        uint32_t o[32];
+        tmem_ld32(t_O + q * 32, o);
+        tc_wait_ld();
+        if (n < p.L) {
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            uint4 vv;
+            vv.x = pack_bf16x2(__uint_as_float(o[8 * i + 0]) * inv_l, __uint_as_float(o[8 * i + 1]) * inv_l);
+            vv.y = pack_bf16x2(__uint_as_float(o[8 * i + 2]) * inv_l, __uint_as_float(o[8 * i + 3]) * inv_l);
+            vv.z = pack_bf16x2(__uint_as_float(o[8 * i + 4]) * inv_l, __uint_as_float(o[8 * i + 5]) * inv_l);
+            vv.w = pack_bf16x2(__uint_as_float(o[8 * i + 6]) * inv_l, __uint_as_float(o[8 * i + 7]) * inv_l);
+            dst[q * 4 + i] = vv;
+          }
         }
-        tc_commit(bar_o);
       }
-    }
-    if (!w.wait(bar_o, ph)) { ok = false; break; }
-    tc_fence_after();
-    if (tid == 0 && j + 1 < total_tiles) {  // V tile is consumed: prefetch the next one
-      issue_kv_load(sV, &tm_v, bar_v, j + 1);
-      v_inflight = true;
+      tc_fence_before();
     }
   }
 
-  // ---- epilogue: O / l -> bf16 -> out[b][n][h][:] -------------------------
-  if (!*abort_flag) {
-    const int n = n0 + tid;
-    const float inv_l = 1.f / l_run;
-    uint4* dst = reinterpret_cast<uint4*>(out + ((static_cast<int64_t>(b) * p.L + n) * p.Hn + h) * kHeadDim);
-#pragma unroll
-    for (int c = 0; c < 4; ++c) {
-      uint32_t o[32];
-      tmem_ld32(t_O + c * 32, o);
-      tc_wait_ld();
-      if (n < p.L) {
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          uint4 vv;
-          vv.x = pack_bf16x2(__uint_as_float(o[8 * i + 0]) * inv_l, __uint_as_float(o[8 * i + 1]) * inv_l);
-          vv.y = pack_bf16x2(__uint_as_float(o[8 * i + 2]) * inv_l, __uint_as_float(o[8 * i + 3]) * inv_l);
-          vv.z = pack_bf16x2(__uint_as_float(o[8 * i + 4]) * inv_l, __uint_as_float(o[8 * i + 5]) * inv_l);
-          vv.w = pack_bf16x2(__uint_as_float(o[8 * i + 6]) * inv_l, __uint_as_float(o[8 * i + 7]) * inv_l);
-          dst[c * 4 + i] = vv;
-        }
-      }
-    }
-  } else if (tid == 0) {
-    // gave up: let this CTA's own copies land (bounded) before the shared memory is released
-    const long long t0 = clock64();
-    while (clock64() - t0 < 2000000LL) {
-      const bool q_done = !q_inflight || mbar_try_wait(bar_q, 0);
-      const bool k_done = !k_inflight || mbar_try_wait(bar_k, 0) || mbar_try_wait(bar_k, 1);
-      const bool v_done = !v_inflight || mbar_try_wait(bar_v, 0) || mbar_try_wait(bar_v, 1);
-      if (q_done && k_done && v_done) break;
-    }
-  }
+  // ---- teardown: every role ends here, also after a timed-out wait --------------------
   tc_fence_before();
   __syncthreads();
-  if (warp == 0) tmem_dealloc(tmem_base, kTmemCols);
+  if (warp == 10 && lane == 0 && *abort_flag) {
+    // gave up: let copies that are still in flight land (bounded) before smem is released
+    const long long t0 = clock64();
+    while (clock64() - t0 < 4000000LL) {
+    }
+  }
+  __syncthreads();
+  if (warp == 8) tmem_dealloc(tmem_base, kTmemCols);
 }
 
 // --------------------------------------------------------------------------
@@ -311,7 +550,27 @@ static bool make_map(CUtensorMap* m, const void* base, int rank, const uint64_t*
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-constexpr int kAttnSmemBytes = 3 * kTileBytes + 1024 + 128;
+struct DeviceInfo {
+  bool ok = false;
+  int sm_count = 0;
+};
+
+static const DeviceInfo& device_info() {
+  static thread_local int cached_dev = -1;
+  static thread_local DeviceInfo info;
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) {
+    info.ok = false;
+    return info;
+  }
+  if (dev != cached_dev) {
+    info.ok = cudaDeviceGetAttribute(&info.sm_count, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess &&
+              cudaFuncSetAttribute(window_attn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                   kAttnSmemBytes) == cudaSuccess;
+    cached_dev = dev;
+  }
+  return info;
+}
 
 }  // namespace unstep
 
@@ -334,14 +593,8 @@ extern "C" int unstep_window_attn(const unstep_shape_t* shape, const int32_t* st
       return UNSTEP_ERR_INVALID_ARG;
   rc = check_device();
   if (rc != UNSTEP_OK) return rc;
-
-  static std::once_flag attr_once;
-  static bool attr_ok = false;
-  std::call_once(attr_once, [] {
-    attr_ok = cudaFuncSetAttribute(window_attn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                   kAttnSmemBytes) == cudaSuccess;
-  });
-  if (!attr_ok) return UNSTEP_ERR_CUDA;
+  const DeviceInfo& info = device_info();
+  if (!info.ok) return UNSTEP_ERR_CUDA;
 
   const uint64_t Hn = shape->heads, C = shape->ring_frames;
   const uint64_t T = static_cast<uint64_t>(shape->grid_h) * shape->grid_w;
@@ -355,11 +608,14 @@ extern "C" int unstep_window_attn(const unstep_shape_t* shape, const int32_t* st
   p.T = static_cast<int32_t>(T);
   p.C = shape->ring_frames;
   p.q_tiles = static_cast<int32_t>((L + kTileM - 1) / kTileM);
+  p.q_pairs = (p.q_tiles + 1) / 2;
   p.tiles_per_frame = static_cast<int32_t>((T + kTileN - 1) / kTileN);
+  p.tail_valid = static_cast<int32_t>(T) - (p.tiles_per_frame - 1) * kTileN;
   p.scale_log2e = 1.4426950408889634f / sqrtf(static_cast<float>(kHeadDim));
 
   for (int b0 = 0; b0 < shape->batch; b0 += kMaxStreamsPerLaunch) {
     const int nb = shape->batch - b0 < kMaxStreamsPerLaunch ? shape->batch - b0 : kMaxStreamsPerLaunch;
+    p.n_streams = nb;
     for (int i = 0; i < nb; ++i) {
       const int hi = start_frame[b0 + i] + shape->chunk_frames;
       const int lo = hi - window_frames > 0 ? hi - window_frames : 0;
@@ -379,13 +635,22 @@ extern "C" int unstep_window_attn(const unstep_shape_t* shape, const int32_t* st
     if (!make_map(&tm_q, qb, 4, qdims, qstr, 2) || !make_map(&tm_k, kb, 5, rdims, rstr, 2) ||
         !make_map(&tm_v, vb, 5, rdims, rstr, 2))
       return UNSTEP_ERR_CUDA;
-    const unsigned grid = static_cast<unsigned>(nb) * p.Hn * p.q_tiles;
-    window_attn_kernel<<<grid, 128, kAttnSmemBytes, st>>>(tm_q, tm_k, tm_v, p, ob);
+    const long long items = static_cast<long long>(nb) * p.Hn * p.q_pairs;
+    const unsigned grid = static_cast<unsigned>(items < info.sm_count ? items : info.sm_count);
+    window_attn_kernel<<<grid, kThreads, kAttnSmemBytes, st>>>(tm_q, tm_k, tm_v, p, ob);
     g_launches.fetch_add(1);
     if (cudaGetLastError() != cudaSuccess) return UNSTEP_ERR_CUDA;
   }
   return UNSTEP_OK;
 }
+
+#ifdef UNSTEP_TRACE
+extern "C" int unstep_debug_read_trace(long long* host_out) {
+  if (cudaDeviceSynchronize() != cudaSuccess) return UNSTEP_ERR_CUDA;
+  return cudaMemcpyFromSymbol(host_out, g_trace, sizeof(long long) * 4 * 64 * 8) == cudaSuccess
+             ? UNSTEP_OK : UNSTEP_ERR_CUDA;
+}
+#endif
 
 extern "C" int unstep_poll_status(void) {
   if (cudaDeviceSynchronize() != cudaSuccess) return UNSTEP_ERR_CUDA;
