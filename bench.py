@@ -56,7 +56,7 @@ class ClockSampler(threading.Thread):
     def __init__(self, index: int, period_s: float = 0.02):
         super().__init__(daemon=True)
         self.index, self.period = index, period_s
-        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self.samples, self.power, self.reasons, self.max_mhz = [], [], set(), None
         self._halt = threading.Event()
         self.error = None
 
@@ -75,6 +75,7 @@ class ClockSampler(threading.Thread):
             }
             while not self._halt.is_set():
                 self.samples.append(int(nv.nvmlDeviceGetClockInfo(h, nv.NVML_CLOCK_SM)))
+                self.power.append(nv.nvmlDeviceGetPowerUsage(h) / 1000.0)
                 mask = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(h))
                 for bit, name in names.items():
                     if mask & bit:
@@ -88,7 +89,8 @@ class ClockSampler(threading.Thread):
         self.join(timeout=2.0)
         med = int(np.median(self.samples)) if self.samples else None
         out = {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
-               "samples": len(self.samples)}
+               "samples": len(self.samples),
+               "power_w": round(float(np.median(self.power)), 1) if self.power else None}
         if self.error:
             out["error"] = self.error
         return out

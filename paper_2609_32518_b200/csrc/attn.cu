@@ -17,7 +17,9 @@
 #include <cuda.h>
 #include <cuda_bf16.h>
 
+#include <map>
 #include <mutex>
+#include <utility>
 
 #include "common.h"
 #include "ptx.cuh"
@@ -64,38 +66,75 @@ struct AttnParams {
   int32_t tail_valid;       // valid keys in the last tile of a frame, 1..128
   int32_t n_streams;
   float scale_log2e;        // log2(e) / sqrt(128)
+  int32_t items_per_stream; // Hn * q_pairs
+  int64_t total_steps;      // sum over items of their key tiles
+  float* part;              // workspace: partial results of split items, kPartFloats per slot
+  int* counters;            // workspace: arrivals per (item, query tile), zero between launches
   int32_t first_frame[kMaxStreamsPerLaunch];  // first attended absolute frame of stream b
   int32_t n_frames[kMaxStreamsPerLaunch];     // attended frames of stream b
+  int64_t step_base[kMaxStreamsPerLaunch];    // steps of all streams before b
 };
+
+// Partial result of one query tile of a split item: O[col][row] (unnormalised, relative to the
+// part's own reference maximum), then m[row], l[row].  Two tiles per slot, two slots per CTA.
+constexpr int kPartTileFloats = 128 * 128 + 2 * 128;
+constexpr int kPartFloats = 2 * kPartTileFloats;
+constexpr int kMinStepsPerCta = 4;
 
 // One unit of work of a CTA: key tiles [t0, t1) of item (b, h, query-tile pair qp).
 struct Seg {
   int b, h, qp, nq, t0, t1;
+  int tiles;          // key tiles of the whole item
+  int item;           // item index inside the launch
+  int64_t item_step0; // global step index of the item's first tile
+  bool first_in_cta;  // this segment starts the CTA's range
 };
 
-// Contiguous, balanced split of the items over the CTAs.  Items are ordered stream, head,
-// query pair, so CTAs that run side by side read the same head's K/V through L2.
+// The (item, key tile) steps of the launch form one sequence, ordered stream, head, query
+// pair, key tile, and every CTA takes an equal contiguous share of it.  An item that straddles
+// a CTA boundary is split along its keys; the parts are merged by whichever CTA finishes last.
+// Neighbouring CTAs work on the same head, so its K/V is shared through L2.
 struct Sched {
-  int cur, end;
+  int64_t lo, hi, cur;
   const AttnParams& p;
+  __device__ static int64_t cta_lo(const AttnParams& p, int64_t c) { return p.total_steps * c / gridDim.x; }
+  __device__ static int cta_of(const AttnParams& p, int64_t step) {
+    int64_t c = step * gridDim.x / p.total_steps;
+    while (c + 1 < gridDim.x && cta_lo(p, c + 1) <= step) ++c;
+    while (c > 0 && cta_lo(p, c) > step) --c;
+    return static_cast<int>(c);
+  }
   __device__ Sched(const AttnParams& prm) : p(prm) {
-    const long long items = static_cast<long long>(p.n_streams) * p.Hn * p.q_pairs;
-    cur = static_cast<int>(items * blockIdx.x / gridDim.x);
-    end = static_cast<int>(items * (blockIdx.x + 1) / gridDim.x);
+    lo = cta_lo(p, blockIdx.x);
+    hi = cta_lo(p, blockIdx.x + 1);
+    cur = lo;
   }
   __device__ bool next(Seg& s) {
-    if (cur >= end) return false;
-    int it = cur++;
-    s.qp = it % p.q_pairs;
-    it /= p.q_pairs;
-    s.h = it % p.Hn;
-    s.b = it / p.Hn;
+    if (cur >= hi) return false;
+    int b = 0;
+    while (b + 1 < p.n_streams && p.step_base[b + 1] <= cur) ++b;
+    const int tiles = p.n_frames[b] * p.tiles_per_frame;
+    const int64_t rel = cur - p.step_base[b];
+    const int in_stream = static_cast<int>(rel / tiles);
+    s.b = b;
+    s.tiles = tiles;
+    s.t0 = static_cast<int>(rel - static_cast<int64_t>(in_stream) * tiles);
+    const int64_t left = hi - cur;
+    s.t1 = (left < tiles - s.t0) ? s.t0 + static_cast<int>(left) : tiles;
+    s.item = b * p.items_per_stream + in_stream;
+    s.item_step0 = cur - s.t0;
+    s.qp = in_stream % p.q_pairs;
+    s.h = in_stream / p.q_pairs;
     s.nq = (2 * s.qp + 1 < p.q_tiles) ? 2 : 1;
-    s.t0 = 0;
-    s.t1 = p.n_frames[s.b] * p.tiles_per_frame;
+    s.first_in_cta = (cur == lo);
+    cur += s.t1 - s.t0;
     return true;
   }
 };
+
+__device__ __forceinline__ void named_barrier_128(int id) {
+  asm volatile("bar.sync %0, 128;" ::"r"(id) : "memory");
+}
 
 struct Waiter {
   volatile int* abort_flag;
@@ -201,7 +240,11 @@ __device__ __forceinline__ bool softmax_tile(uint32_t t_S, uint32_t t_O, float c
                                                __uint_as_float(sreg[64 * half + 2 * i + 1])), c2, nm2);
       float x0, x1;
       unpack_f32x2(x2, x0, x1);
+#ifdef X_NOEXP
+      const float p0 = x0 * 1e-3f, p1 = x1 * 1e-3f;
+#else
       const float p0 = ex2(x0), p1 = ex2(x1);
+#endif
       acc[i & 3] = add_f32x2(acc[i & 3], pack_f32x2(p0, p1));
       preg[i] = pack_bf16x2(p0, p1);
     }
@@ -242,6 +285,7 @@ window_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
   const uint32_t bar_turn = bar_o_final + 16;                // [2]  softmax 1-a -> softmax a
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(gen + kSmemBar + 192);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(gen + kSmemBar + 200);
+  volatile int* merge_flag = reinterpret_cast<volatile int*>(gen + kSmemBar + 208);  // [2]
 
   const int tid = threadIdx.x;
   const int warp = tid >> 5;
@@ -466,29 +510,96 @@ window_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         if (paired) ++pair_it;
       }
       if (!ok) break;
-      // epilogue: wait for the last P V, then O / l -> bf16 -> out[b][n][h][:]
+      // epilogue: wait for the last P V of the segment
       ok = w.wait(my_o_final, seg_it & 1);
       if (!ok) break;
       ++seg_it;
       tc_fence_after();
       const int n = (2 * s.qp + a) * kTileM + row;
-      const float inv_l = 1.f / l_run;
       uint4* dst = reinterpret_cast<uint4*>(
           out + ((static_cast<int64_t>(s.b) * p.L + n) * p.Hn + s.h) * kHeadDim);
+      const bool whole = (s.t0 == 0 && s.t1 == s.tiles);
+      if (whole) {
+        // O / l -> bf16 -> out[b][n][h][:]
+        const float inv_l = 1.f / l_run;
 #pragma unroll
-      for (int q = 0; q < 4; ++q) {
-        uint32_t o[32];
-        tmem_ld32(t_O + q * 32, o);
-        tc_wait_ld();
-        if (n < p.L) {
+        for (int q = 0; q < 4; ++q) {
+          uint32_t o[32];
+          tmem_ld32(t_O + q * 32, o);
+          tc_wait_ld();
+          if (n < p.L) {
 #pragma unroll
-          for (int i = 0; i < 4; ++i) {
-            uint4 vv;
-            vv.x = pack_bf16x2(__uint_as_float(o[8 * i + 0]) * inv_l, __uint_as_float(o[8 * i + 1]) * inv_l);
-            vv.y = pack_bf16x2(__uint_as_float(o[8 * i + 2]) * inv_l, __uint_as_float(o[8 * i + 3]) * inv_l);
-            vv.z = pack_bf16x2(__uint_as_float(o[8 * i + 4]) * inv_l, __uint_as_float(o[8 * i + 5]) * inv_l);
-            vv.w = pack_bf16x2(__uint_as_float(o[8 * i + 6]) * inv_l, __uint_as_float(o[8 * i + 7]) * inv_l);
-            dst[q * 4 + i] = vv;
+            for (int i = 0; i < 4; ++i) {
+              uint4 vv;
+              vv.x = pack_bf16x2(__uint_as_float(o[8 * i + 0]) * inv_l, __uint_as_float(o[8 * i + 1]) * inv_l);
+              vv.y = pack_bf16x2(__uint_as_float(o[8 * i + 2]) * inv_l, __uint_as_float(o[8 * i + 3]) * inv_l);
+              vv.z = pack_bf16x2(__uint_as_float(o[8 * i + 4]) * inv_l, __uint_as_float(o[8 * i + 5]) * inv_l);
+              vv.w = pack_bf16x2(__uint_as_float(o[8 * i + 6]) * inv_l, __uint_as_float(o[8 * i + 7]) * inv_l);
+              dst[q * 4 + i] = vv;
+            }
+          }
+        }
+      } else {
+        // part of a split item: publish (O, m, l), count the arrival; the last part to arrive
+        // merges all of them in part order (a fixed order, so the result does not depend on
+        // which CTA happens to be last)
+        float* mine = p.part + (static_cast<int64_t>(2 * blockIdx.x + (s.first_in_cta ? 0 : 1)) * kPartFloats +
+                                a * kPartTileFloats);
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          uint32_t o[32];
+          tmem_ld32(t_O + q * 32, o);
+          tc_wait_ld();
+#pragma unroll
+          for (int i = 0; i < 32; ++i) mine[(q * 32 + i) * 128 + row] = __uint_as_float(o[i]);
+        }
+        mine[128 * 128 + row] = m_run;
+        mine[128 * 128 + 128 + row] = l_run;
+        __threadfence();
+        named_barrier_128(1 + a);
+        const int c_lo = Sched::cta_of(p, s.item_step0);
+        const int c_hi = Sched::cta_of(p, s.item_step0 + s.tiles - 1);
+        if (row == 0) merge_flag[a] = atomicAdd(p.counters + 2 * s.item + a, 1);
+        named_barrier_128(1 + a);
+        if (merge_flag[a] == c_hi - c_lo) {
+          if (row == 0) p.counters[2 * s.item + a] = 0;  // ready for the next launch
+          __threadfence();
+          auto part_of = [&](int c) -> const float* {
+            const int64_t clo = Sched::cta_lo(p, c);
+            const bool first = clo >= s.item_step0;   // the part starts the range of CTA c
+            return p.part + (static_cast<int64_t>(2 * c + (first ? 0 : 1)) * kPartFloats + a * kPartTileFloats);
+          };
+          float m_all = -INFINITY;
+          for (int c = c_lo; c <= c_hi; ++c) m_all = fmaxf(m_all, __ldcg(part_of(c) + 128 * 128 + row));
+          float l_all = 0.f;
+          for (int c = c_lo; c <= c_hi; ++c) {
+            const float* pc = part_of(c);
+            l_all += __ldcg(pc + 128 * 128 + 128 + row) *
+                     ex2((__ldcg(pc + 128 * 128 + row) - m_all) * p.scale_log2e);
+          }
+          const float inv_l = 1.f / l_all;
+#pragma unroll 1
+          for (int q = 0; q < 4; ++q) {
+            float acc[32];
+#pragma unroll
+            for (int i = 0; i < 32; ++i) acc[i] = 0.f;
+            for (int c = c_lo; c <= c_hi; ++c) {
+              const float* pc = part_of(c);
+              const float sc = ex2((__ldcg(pc + 128 * 128 + row) - m_all) * p.scale_log2e);
+#pragma unroll
+              for (int i = 0; i < 32; ++i) acc[i] = fmaf(__ldcg(pc + (q * 32 + i) * 128 + row), sc, acc[i]);
+            }
+            if (n < p.L) {
+#pragma unroll
+              for (int i = 0; i < 4; ++i) {
+                uint4 vv;
+                vv.x = pack_bf16x2(acc[8 * i + 0] * inv_l, acc[8 * i + 1] * inv_l);
+                vv.y = pack_bf16x2(acc[8 * i + 2] * inv_l, acc[8 * i + 3] * inv_l);
+                vv.z = pack_bf16x2(acc[8 * i + 4] * inv_l, acc[8 * i + 5] * inv_l);
+                vv.w = pack_bf16x2(acc[8 * i + 6] * inv_l, acc[8 * i + 7] * inv_l);
+                dst[q * 4 + i] = vv;
+              }
+            }
           }
         }
       }
@@ -572,6 +683,51 @@ static const DeviceInfo& device_info() {
   return info;
 }
 
+// Scratch for split items, one per (device, stream): calls on one stream run in order and may
+// share it; calls on different streams may overlap on the GPU and must not.  Allocated on first
+// use and kept; it only grows.
+struct Workspace {
+  float* part = nullptr;
+  int* counters = nullptr;
+  size_t slots = 0, n_counters = 0;
+};
+static std::mutex g_ws_mutex;
+static std::map<std::pair<int, cudaStream_t>, Workspace> g_workspaces;
+
+static bool get_workspace(cudaStream_t st, size_t slots, size_t n_counters, Workspace* out) {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return false;
+  std::lock_guard<std::mutex> lock(g_ws_mutex);
+  Workspace& ws = g_workspaces[std::make_pair(dev, st)];
+  if (ws.slots < slots) {
+    if (ws.part != nullptr && cudaFree(ws.part) != cudaSuccess) return false;
+    ws.part = nullptr;
+    ws.slots = 0;
+    if (cudaMalloc(&ws.part, slots * kPartFloats * sizeof(float)) != cudaSuccess) return false;
+    ws.slots = slots;
+  }
+  if (ws.n_counters < n_counters) {
+    if (ws.counters != nullptr && cudaFree(ws.counters) != cudaSuccess) return false;
+    ws.counters = nullptr;
+    ws.n_counters = 0;
+    if (cudaMalloc(&ws.counters, n_counters * sizeof(int)) != cudaSuccess) return false;
+    if (cudaMemset(ws.counters, 0, n_counters * sizeof(int)) != cudaSuccess) return false;
+    ws.n_counters = n_counters;
+  }
+  *out = ws;
+  return true;
+}
+
+// After a kernel gave up, arrival counters may be left non-zero: clear them all.
+static void reset_workspace_counters() {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return;
+  std::lock_guard<std::mutex> lock(g_ws_mutex);
+  for (auto& kv : g_workspaces)
+    if (kv.first.first == dev && kv.second.counters != nullptr)
+      cudaMemset(kv.second.counters, 0, kv.second.n_counters * sizeof(int));
+}
+
 }  // namespace unstep
 
 using namespace unstep;
@@ -612,6 +768,7 @@ extern "C" int unstep_window_attn(const unstep_shape_t* shape, const int32_t* st
   p.tiles_per_frame = static_cast<int32_t>((T + kTileN - 1) / kTileN);
   p.tail_valid = static_cast<int32_t>(T) - (p.tiles_per_frame - 1) * kTileN;
   p.scale_log2e = 1.4426950408889634f / sqrtf(static_cast<float>(kHeadDim));
+  p.items_per_stream = p.Hn * p.q_pairs;
 
   for (int b0 = 0; b0 < shape->batch; b0 += kMaxStreamsPerLaunch) {
     const int nb = shape->batch - b0 < kMaxStreamsPerLaunch ? shape->batch - b0 : kMaxStreamsPerLaunch;
@@ -622,6 +779,21 @@ extern "C" int unstep_window_attn(const unstep_shape_t* shape, const int32_t* st
       p.first_frame[i] = lo;
       p.n_frames[i] = hi - lo;
     }
+    int64_t steps = 0;
+    for (int i = 0; i < nb; ++i) {
+      p.step_base[i] = steps;
+      steps += static_cast<int64_t>(p.items_per_stream) * p.n_frames[i] * p.tiles_per_frame;
+    }
+    p.total_steps = steps;
+    int64_t want = steps / kMinStepsPerCta;
+    if (want < 1) want = 1;
+    const unsigned grid = static_cast<unsigned>(want < info.sm_count ? want : info.sm_count);
+    Workspace ws;
+    if (!get_workspace(st, 2 * static_cast<size_t>(grid),
+                       2 * static_cast<size_t>(nb) * p.items_per_stream, &ws))
+      return UNSTEP_ERR_CUDA;
+    p.part = ws.part;
+    p.counters = ws.counters;
     const char* qb = static_cast<const char*>(q_rot) + static_cast<uint64_t>(b0) * L * row_bytes;
     const char* kb = static_cast<const char*>(ring_k) + static_cast<uint64_t>(b0) * C * T * row_bytes;
     const char* vb = static_cast<const char*>(ring_v) + static_cast<uint64_t>(b0) * C * T * row_bytes;
@@ -635,8 +807,6 @@ extern "C" int unstep_window_attn(const unstep_shape_t* shape, const int32_t* st
     if (!make_map(&tm_q, qb, 4, qdims, qstr, 2) || !make_map(&tm_k, kb, 5, rdims, rstr, 2) ||
         !make_map(&tm_v, vb, 5, rdims, rstr, 2))
       return UNSTEP_ERR_CUDA;
-    const long long items = static_cast<long long>(nb) * p.Hn * p.q_pairs;
-    const unsigned grid = static_cast<unsigned>(items < info.sm_count ? items : info.sm_count);
     window_attn_kernel<<<grid, kThreads, kAttnSmemBytes, st>>>(tm_q, tm_k, tm_v, p, ob);
     g_launches.fetch_add(1);
     if (cudaGetLastError() != cudaSuccess) return UNSTEP_ERR_CUDA;
@@ -656,6 +826,9 @@ extern "C" int unstep_poll_status(void) {
   if (cudaDeviceSynchronize() != cudaSuccess) return UNSTEP_ERR_CUDA;
   int st = 0, zero = 0;
   if (cudaMemcpyFromSymbol(&st, g_status, sizeof(int)) != cudaSuccess) return UNSTEP_ERR_CUDA;
-  if (st != 0 && cudaMemcpyToSymbol(g_status, &zero, sizeof(int)) != cudaSuccess) return UNSTEP_ERR_CUDA;
+  if (st != 0) {
+    if (cudaMemcpyToSymbol(g_status, &zero, sizeof(int)) != cudaSuccess) return UNSTEP_ERR_CUDA;
+    reset_workspace_counters();
+  }
   return st;
 }
