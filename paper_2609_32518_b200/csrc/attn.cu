@@ -1,8 +1,8 @@
 // Windowed attention of one chunk over the KV ring (sm_100a).
 //
 // Persistent, warp-specialised kernel, one CTA per SM:
-//   warps 0-3   softmax of query tile 0 (one thread per query row)
-//   warps 4-7   softmax of query tile 1
+//   warps 0-7   softmax: two threads per query row (64 key columns each); the eight warps
+//               work on one query tile at a time and alternate between the item's two tiles
 //   warp  8, 9  tcgen05.mma issuers of query tile 0 and 1 (one lane each); warp 8 owns TMEM
 //   warp  10    TMA producer (one lane)
 // A work item is (stream, head, pair of 128-query tiles): both tiles share every K/V
@@ -35,7 +35,7 @@ __device__ int g_status = 0;
 __device__ long long g_trace[4][64][8];
 #define TRACE(role, tile, ev)                                                          \
   do {                                                                                 \
-    if (blockIdx.x == 0 && (tile) < 64 && (threadIdx.x & 31) == 0 && ((threadIdx.x >> 5) & 3) < 2 && (threadIdx.x < 128 ? threadIdx.x == 0 : true) && (threadIdx.x >= 256 || (threadIdx.x & 127) == 0)) g_trace[role][tile][ev] = clock64(); \
+    if (blockIdx.x == 0 && (tile) < 64 && (threadIdx.x == 0 || threadIdx.x == 256 || threadIdx.x == 288)) g_trace[role][tile][ev] = clock64(); \
   } while (0)
 #else
 #define TRACE(role, tile, ev) \
@@ -56,7 +56,8 @@ constexpr float kRescaleThreshold = 8.f;    // log2 units: rescale O only when t
 constexpr int kSmemQ = 0;
 constexpr int kSmemKV = 2 * kTileBytes;
 constexpr int kSmemBar = kSmemKV + kStages * kTileBytes;
-constexpr int kAttnSmemBytes = kSmemBar + 256 + 1024;  // + barriers/flags + alignment slack
+constexpr int kSmemXchg = kSmemBar + 256;                // float[2][2][128]: row max / row sum exchange
+constexpr int kAttnSmemBytes = kSmemXchg + 2048;
 
 struct AttnParams {
   int32_t Hn, L, T, C;
@@ -161,47 +162,83 @@ __device__ __forceinline__ void reg_dealloc_96() { asm volatile("setmaxnreg.dec.
 __device__ __forceinline__ void reg_alloc_200() { asm volatile("setmaxnreg.inc.sync.aligned.u32 200;"); }
 
 // --------------------------------------------------------------------------------------
-// Softmax of one 128 x 128 score tile for this thread's row.
-//   t_S / t_O  : TMEM addresses (this warp's lanes) of the score and output tiles
-//   kMasked    : columns >= nvalid are excluded (last tile of a frame)
-// The running maximum is only raised when it grows by more than 2^kRescaleThreshold, so
-// the output accumulator is rescaled rarely; P stays below 2^8 in between.  The caller has
-// seen S of this tile complete, which (the tensor pipe runs in issue order) also means the
-// previous P V into O has landed, so O may be rescaled here without another wait.
-// P is handed to the MMA warp in two halves of 64 keys (bar_p_half, bar_p_half + 8).
-// The two warpgroups take turns on the exponentials (bar_turn_wait / bar_turn_signal, 0 = no
-// partner): the MUFU pipe is shared, and alternating keeps the two query tiles half a period
-// apart, so that the tensor pipe always has one tile's MMAs to run while the other tile is
-// in its softmax.  Returns false when a bounded wait gave up.
+// Softmax of one 128 x 128 score tile.  All eight softmax warps work on the same tile: the
+// thread pair (warp w, warp w + 4) shares a query row, each taking 64 of its 128 key columns,
+// and the warps alternate between the two query tiles of the item.  So the exponentials of one
+// tile run on all four MUFU pipes at once, its P reaches the tensor core sooner, and while the
+// tensor core works on that tile the warps are busy with the other one.
+//   t_S / t_O : TMEM addresses (this warp's lanes) of the tile's scores and output
+//   half      : which 64 columns this thread owns
+//   xchg      : shared float[2][128] used to combine the two partial row maxima
+//   kMasked   : key columns >= nvalid are excluded (last tile of a frame)
+// The running maximum is only raised when it grows by more than 2^kRescaleThreshold, so the
+// output accumulator is rescaled rarely; P stays below 2^8 in between.  Both threads of a row
+// take the same decision from the same combined maximum.  The caller has seen S of this tile
+// complete, which (the tensor pipe runs in issue order) also means the previous P V into O has
+// landed, so O may be rescaled here without another wait.
+// P (bf16 pairs) overwrites the first 64 columns of S: this thread's 32 columns are written
+// only after the row's partner has loaded its scores (the barrier of the max exchange).
 // --------------------------------------------------------------------------------------
+__device__ __forceinline__ void softmax_barrier() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
+
 template <bool kMasked>
 __device__ __forceinline__ bool softmax_tile(uint32_t t_S, uint32_t t_O, float c, int nvalid,
-                                             bool first, float& m_run, float& l_run,
-                                             uint32_t bar_p_half, const Waiter& w,
-                                             uint32_t bar_turn_wait, uint32_t turn_parity,
-                                             uint32_t bar_turn_signal, int trace_role,
-                                             int trace_tile) {
-  uint32_t sreg[128];
+                                             bool first, int half, int row, volatile float* xchg,
+                                             volatile int* abort_flag, float& m_run, float& l_run,
+                                             uint32_t bar_p, int trace_role, int trace_tile) {
+  uint32_t sreg[64];
+#ifdef X_NOLD
 #pragma unroll
-  for (int q = 0; q < 4; ++q) tmem_ld32(t_S + q * 32, sreg + q * 32);
+  for (int i = 0; i < 64; ++i) sreg[i] = 0x3f800000u + i + row;
+#else
+  tmem_ld32(t_S + 64 * half, sreg);
+  tmem_ld32(t_S + 64 * half + 32, sreg + 32);
   tc_wait_ld();
+#endif
   TRACE(trace_role, trace_tile, 2);
+#ifdef X_NOSOFTMAX
+  {
+    xchg[half * 128 + row] = 0.f;
+    softmax_barrier();
+    if (*abort_flag) return false;
+    uint32_t preg[32];
+#pragma unroll
+    for (int i = 0; i < 32; ++i) preg[i] = sreg[i] ^ sreg[i + 32];
+#ifndef X_NOLD
+    tmem_st32(t_S + 32 * half, preg);
+    tc_wait_st();
+#else
+    if (preg[0] == 0x12345u) l_run += 1.f;
+#endif
+    tc_fence_before();
+    mbar_arrive(bar_p);
+    l_run += 1.f;
+    m_run = 0.f;
+    return true;
+  }
+#endif
   if (kMasked) {
 #pragma unroll
-    for (int i = 0; i < 128; ++i)
-      if (i >= nvalid) sreg[i] = 0xFF800000u;  // -inf
+    for (int i = 0; i < 64; ++i)
+      if (64 * half + i >= nvalid) sreg[i] = 0xFF800000u;  // -inf
   }
-  // row maximum: four independent chains of 3-input max
-  float mx4[4];
+  // partial row maximum: two independent chains of 3-input max
+  float mx2[2];
 #pragma unroll
-  for (int q = 0; q < 4; ++q) {
+  for (int q = 0; q < 2; ++q) {
     float m = fmaxf(__uint_as_float(sreg[32 * q]), __uint_as_float(sreg[32 * q + 1]));
 #pragma unroll
     for (int i = 2; i < 32; i += 2)
       m = max3(m, __uint_as_float(sreg[32 * q + i]), __uint_as_float(sreg[32 * q + i + 1]));
-    mx4[q] = m;
+    mx2[q] = m;
   }
-  const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
+  float mx = fmaxf(mx2[0], mx2[1]);
+  xchg[half * 128 + row] = mx;
+  softmax_barrier();
+  // a thread whose wait gave up still comes to the barrier (nobody is left waiting there);
+  // the flag it raised before is visible to all now, and all leave together
+  if (*abort_flag) return false;
+  mx = fmaxf(mx, xchg[(1 - half) * 128 + row]);
   TRACE(trace_role, trace_tile, 3);
   float alpha = 1.f;
   bool grow = false;
@@ -215,46 +252,40 @@ __device__ __forceinline__ bool softmax_tile(uint32_t t_S, uint32_t t_O, float c
   }
   if (__any_sync(0xFFFFFFFFu, grow)) {
 #pragma unroll
-    for (int q = 0; q < 4; ++q) {
+    for (int q = 0; q < 2; ++q) {
       uint32_t o[32];
-      tmem_ld32(t_O + q * 32, o);
+      tmem_ld32(t_O + 64 * half + q * 32, o);
       tc_wait_ld();
 #pragma unroll
       for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
-      tmem_st32(t_O + q * 32, o);
+      tmem_st32(t_O + 64 * half + q * 32, o);
     }
   }
-  if (bar_turn_wait != 0u && !w.wait(bar_turn_wait, turn_parity)) return false;
-  TRACE(trace_role, trace_tile, 6);
   // p = 2^(s*c - m*c): packed FMA on pairs, one MUFU per element, packed partial sums
   const uint64_t c2 = pack_f32x2(c, c);
   const float neg_ms = -m_run * c;
   const uint64_t nm2 = pack_f32x2(neg_ms, neg_ms);
   uint64_t acc[4] = {0ull, 0ull, 0ull, 0ull};
+  uint32_t preg[32];
 #pragma unroll
-  for (int half = 0; half < 2; ++half) {
-    uint32_t preg[32];
-#pragma unroll
-    for (int i = 0; i < 32; ++i) {
-      const uint64_t x2 = fma_f32x2(pack_f32x2(__uint_as_float(sreg[64 * half + 2 * i]),
-                                               __uint_as_float(sreg[64 * half + 2 * i + 1])), c2, nm2);
-      float x0, x1;
-      unpack_f32x2(x2, x0, x1);
+  for (int i = 0; i < 32; ++i) {
+    const uint64_t x2 = fma_f32x2(pack_f32x2(__uint_as_float(sreg[2 * i]), __uint_as_float(sreg[2 * i + 1])),
+                                  c2, nm2);
+    float x0, x1;
+    unpack_f32x2(x2, x0, x1);
 #ifdef X_NOEXP
-      const float p0 = x0 * 1e-3f, p1 = x1 * 1e-3f;
+    const float p0 = x0 * 1e-3f, p1 = x1 * 1e-3f;
 #else
-      const float p0 = ex2(x0), p1 = ex2(x1);
+    const float p0 = ex2(x0), p1 = ex2(x1);
 #endif
-      acc[i & 3] = add_f32x2(acc[i & 3], pack_f32x2(p0, p1));
-      preg[i] = pack_bf16x2(p0, p1);
-    }
-    tmem_st32(t_S + 32 * half, preg);  // P (bf16 pairs) overwrites the first 64 columns of S
-    if (half == 1 && bar_turn_signal != 0u) mbar_arrive(bar_turn_signal);
-    tc_wait_st();
-    tc_fence_before();
-    mbar_arrive(bar_p_half + 8 * half);
-    TRACE(trace_role, trace_tile, 4 + half);
+    acc[i & 3] = add_f32x2(acc[i & 3], pack_f32x2(p0, p1));
+    preg[i] = pack_bf16x2(p0, p1);
   }
+  tmem_st32(t_S + 32 * half, preg);
+  tc_wait_st();
+  tc_fence_before();
+  mbar_arrive(bar_p);
+  TRACE(trace_role, trace_tile, 4);
   {
     const uint64_t t = add_f32x2(add_f32x2(acc[0], acc[1]), add_f32x2(acc[2], acc[3]));
     float t0, t1;
@@ -268,9 +299,13 @@ __global__ void __launch_bounds__(kThreads, 1)
 window_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                    const __grid_constant__ CUtensorMap tm_v, const AttnParams p,
                    __nv_bfloat16* __restrict__ out) {
-  extern __shared__ uint8_t smem_raw[];
-  const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-  uint8_t* gen = smem_raw + (smem_base - smem_u32(smem_raw));
+  extern __shared__ __align__(1024) uint8_t smem_raw[];
+  const uint32_t smem_base = smem_u32(smem_raw);
+  if (smem_base & 1023u) {  // the 128-byte swizzle needs 1024-byte aligned tiles
+    if (threadIdx.x == 0) atomicExch(&g_status, UNSTEP_ERR_CUDA);
+    return;
+  }
+  uint8_t* gen = smem_raw;
   const uint32_t sQ = smem_base + kSmemQ;
   const uint32_t sKV = smem_base + kSmemKV;
   const uint32_t sBar = smem_base + kSmemBar;
@@ -282,10 +317,10 @@ window_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
   const uint32_t bar_s_full = sBar + 32 + 16 * kStages;      // [2]  MMA warp a -> softmax a
   const uint32_t bar_p_half = bar_s_full + 16;               // [2][2] softmax a -> MMA warp a
   const uint32_t bar_o_final = bar_p_half + 32;              // [2]  MMA warp a -> softmax a
-  const uint32_t bar_turn = bar_o_final + 16;                // [2]  softmax 1-a -> softmax a
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(gen + kSmemBar + 192);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(gen + kSmemBar + 200);
-  volatile int* merge_flag = reinterpret_cast<volatile int*>(gen + kSmemBar + 208);  // [2]
+  volatile int* merge_flag = reinterpret_cast<volatile int*>(gen + kSmemBar + 208);
+  volatile float* xchg = reinterpret_cast<volatile float*>(gen + kSmemXchg);
 
   const int tid = threadIdx.x;
   const int warp = tid >> 5;
@@ -299,7 +334,6 @@ window_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
       mbar_init(bar_p_half + 16 * i, 128);
       mbar_init(bar_p_half + 16 * i + 8, 128);
       mbar_init(bar_o_final + 8 * i, 1);
-      mbar_init(bar_turn + 8 * i, 128);
     }
     for (int i = 0; i < kStages; ++i) {
       mbar_init(bar_kv_full + 8 * i, 1);
@@ -353,9 +387,16 @@ window_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
             if (!ok) break;
             const uint32_t dst = sKV + st * kTileBytes, bar = bar_kv_full + 8 * st;
             const CUtensorMap* tm = kv == 0 ? &tm_k : &tm_v;
+#if defined(X_NOTMA)
+            mbar_arrive(bar);
+#elif defined(X_HALFTMA)
+            mbar_expect_tx(bar, kHalfBytes);
+            tma_load_5d(dst, tm, bar, 0, s.h, tok0, slot_f, s.b);
+#else
             mbar_expect_tx(bar, kTileBytes);
             tma_load_5d(dst, tm, bar, 0, s.h, tok0, slot_f, s.b);
             tma_load_5d(dst + kHalfBytes, tm, bar, 64, s.h, tok0, slot_f, s.b);
+#endif
             ++kv_it;
           }
           if (++ti == p.tiles_per_frame) {
@@ -391,7 +432,9 @@ window_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
 #pragma unroll
         for (int k = 0; k < 8; ++k) {
           const uint64_t off = static_cast<uint64_t>(((k >> 2) * kHalfBytes + (k & 3) * 32) >> 4);
+#ifndef X_NOQK
           mma_ss(s_tmem, dq + off, dk + off, idesc, k > 0);
+#endif
         }
         tc_commit(my_s_full);
         tc_commit(bar_kv_empty + 8 * stage);
@@ -399,7 +442,11 @@ window_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
       auto issue_pv_half = [&](uint64_t dv, int half, int k_steps, bool accumulate) {
 #pragma unroll
         for (int k = 4 * half; k < 4 * half + 4; ++k)
+#ifndef X_NOPV
           if (k < k_steps)
+#else
+          if (k < k_steps && k == 100)
+#endif
             mma_ts(o_tmem, s_tmem + k * 8, dv + static_cast<uint64_t>((k * 2048) >> 4), idesc_pv,
                    (accumulate || k > 0) ? 1u : 0u);
       };
@@ -440,16 +487,15 @@ window_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
           if (part) {
             const uint64_t dv = dv0 + static_cast<uint64_t>((vst * kTileBytes) >> 4);
             TRACE(2 + a, sp_it, 0);
+            // both column halves of P (and any rescale of O) must be in before O is touched
             ok = w.wait(my_p_half, sp_it & 1);
             if (!ok) break;
             TRACE(2 + a, sp_it, 1);
-            tc_fence_after();
-            issue_pv_half(dv, 0, k_steps, j > 0);
-            TRACE(2 + a, sp_it, 2);
             ok = w.wait(my_p_half + 8, sp_it & 1);
             if (!ok) break;
             TRACE(2 + a, sp_it, 3);
             tc_fence_after();
+            issue_pv_half(dv, 0, k_steps, j > 0);
             issue_pv_half(dv, 1, k_steps, true);
             tc_commit(bar_kv_empty + 8 * vst);
             TRACE(2 + a, sp_it, 4);
@@ -469,141 +515,154 @@ window_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
       }
     }
   } else {
-    // ---------------------------------------------------------------- softmax warpgroups
+    // ---------------------------------------------------------------- softmax warps
     reg_alloc_200();
-    const int a = warp >> 2;               // query tile of this warpgroup
+    const int half = warp >> 2;            // which 64 key columns / output columns of the row
     const int row = tid & 127;             // row inside the tile = TMEM lane
     const uint32_t t_lane = tmem_base + (static_cast<uint32_t>((warp & 3) * 32) << 16);
-    const uint32_t t_S = t_lane + a * 128;
-    const uint32_t t_O = t_lane + 256 + a * 128;
-    const uint32_t my_s_full = bar_s_full + 8 * a, my_p_half = bar_p_half + 16 * a,
-                   my_o_final = bar_o_final + 8 * a;
     Sched sched(p);
     Seg s;
-    uint32_t it = 0, seg_it = 0, pair_it = 0;  // pair_it: tiles seen while both warpgroups work
+    uint32_t it[2] = {0, 0}, seg_it[2] = {0, 0}, x_it = 0;
     bool ok = true;
     while (ok && sched.next(s)) {
-      if (a >= s.nq) continue;
-      const bool paired = s.nq == 2;
-      const uint32_t turn_wait = paired ? bar_turn + 8 * a : 0u;
-      const uint32_t turn_signal = paired ? bar_turn + 8 * (1 - a) : 0u;
-      float m_run = -INFINITY, l_run = 0.f;
+      float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};
       int ti = s.t0 % p.tiles_per_frame;
-      for (int j = s.t0; j < s.t1; ++j) {
-        TRACE(a, it, 0);
-        ok = w.wait(my_s_full, it & 1);
-        if (!ok) break;
-        tc_fence_after();
-        TRACE(a, it, 1);
-        const bool tail = (ti == p.tiles_per_frame - 1);
+      for (int j = s.t0; j < s.t1 && ok; ++j) {
+        const bool tail = (ti == p.tiles_per_frame - 1) && p.tail_valid < kTileN;
         if (++ti == p.tiles_per_frame) ti = 0;
-        // tile 0 waits for tile 1's previous tile, tile 1 for tile 0's current one
-        const uint32_t turn_parity = (a == 0) ? ((pair_it & 1) ^ 1) : (pair_it & 1);
-        if (tail && p.tail_valid < kTileN)
-          ok = softmax_tile<true>(t_S, t_O, p.scale_log2e, p.tail_valid, j == s.t0, m_run, l_run, my_p_half,
-                                  w, turn_wait, turn_parity, turn_signal, a, it);
-        else
-          ok = softmax_tile<false>(t_S, t_O, p.scale_log2e, kTileN, j == s.t0, m_run, l_run, my_p_half,
-                                   w, turn_wait, turn_parity, turn_signal, a, it);
-        if (!ok) break;
-        ++it;
-        if (paired) ++pair_it;
+#pragma unroll
+        for (int a = 0; a < 2; ++a) {
+          if (a >= s.nq) break;
+          TRACE(a, it[a], 0);
+          w.wait(bar_s_full + 8 * a, it[a] & 1);  // on failure the flag is up: handled after the barrier
+          tc_fence_after();
+          TRACE(a, it[a], 1);
+          volatile float* xc = xchg + (x_it & 1) * 256;
+          const uint32_t t_S = t_lane + a * 128, t_O = t_lane + 256 + a * 128;
+          const uint32_t bar_p = bar_p_half + 16 * a + 8 * half;
+          if (tail)
+            ok = softmax_tile<true>(t_S, t_O, p.scale_log2e, p.tail_valid, j == s.t0, half, row, xc,
+                                    abort_flag, m_run[a], l_run[a], bar_p, a, it[a]);
+          else
+            ok = softmax_tile<false>(t_S, t_O, p.scale_log2e, kTileN, j == s.t0, half, row, xc,
+                                     abort_flag, m_run[a], l_run[a], bar_p, a, it[a]);
+          if (!ok) break;
+          ++it[a];
+          ++x_it;
+        }
       }
       if (!ok) break;
-      // epilogue: wait for the last P V of the segment
-      ok = w.wait(my_o_final, seg_it & 1);
-      if (!ok) break;
-      ++seg_it;
-      tc_fence_after();
-      const int n = (2 * s.qp + a) * kTileM + row;
-      uint4* dst = reinterpret_cast<uint4*>(
-          out + ((static_cast<int64_t>(s.b) * p.L + n) * p.Hn + s.h) * kHeadDim);
-      const bool whole = (s.t0 == 0 && s.t1 == s.tiles);
-      if (whole) {
-        // O / l -> bf16 -> out[b][n][h][:]
-        const float inv_l = 1.f / l_run;
-#pragma unroll
-        for (int q = 0; q < 4; ++q) {
-          uint32_t o[32];
-          tmem_ld32(t_O + q * 32, o);
-          tc_wait_ld();
-          if (n < p.L) {
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-              uint4 vv;
-              vv.x = pack_bf16x2(__uint_as_float(o[8 * i + 0]) * inv_l, __uint_as_float(o[8 * i + 1]) * inv_l);
-              vv.y = pack_bf16x2(__uint_as_float(o[8 * i + 2]) * inv_l, __uint_as_float(o[8 * i + 3]) * inv_l);
-              vv.z = pack_bf16x2(__uint_as_float(o[8 * i + 4]) * inv_l, __uint_as_float(o[8 * i + 5]) * inv_l);
-              vv.w = pack_bf16x2(__uint_as_float(o[8 * i + 6]) * inv_l, __uint_as_float(o[8 * i + 7]) * inv_l);
-              dst[q * 4 + i] = vv;
-            }
-          }
+      // epilogue of both query tiles
+      for (int a = 0; a < s.nq && ok; ++a) {
+        w.wait(bar_o_final + 8 * a, seg_it[a] & 1);
+        ++seg_it[a];
+        tc_fence_after();
+        // row sum = the two partners' partial sums
+        volatile float* xc = xchg + (x_it & 1) * 256;
+        ++x_it;
+        xc[half * 128 + row] = l_run[a];
+        softmax_barrier();
+        if (*abort_flag) {
+          ok = false;
+          break;
         }
-      } else {
-        // part of a split item: publish (O, m, l), count the arrival; the last part to arrive
-        // merges all of them in part order (a fixed order, so the result does not depend on
-        // which CTA happens to be last)
-        float* mine = p.part + (static_cast<int64_t>(2 * blockIdx.x + (s.first_in_cta ? 0 : 1)) * kPartFloats +
-                                a * kPartTileFloats);
-#pragma unroll
-        for (int q = 0; q < 4; ++q) {
-          uint32_t o[32];
-          tmem_ld32(t_O + q * 32, o);
-          tc_wait_ld();
-#pragma unroll
-          for (int i = 0; i < 32; ++i) mine[(q * 32 + i) * 128 + row] = __uint_as_float(o[i]);
-        }
-        mine[128 * 128 + row] = m_run;
-        mine[128 * 128 + 128 + row] = l_run;
-        __threadfence();
-        named_barrier_128(1 + a);
-        const int c_lo = Sched::cta_of(p, s.item_step0);
-        const int c_hi = Sched::cta_of(p, s.item_step0 + s.tiles - 1);
-        if (row == 0) merge_flag[a] = atomicAdd(p.counters + 2 * s.item + a, 1);
-        named_barrier_128(1 + a);
-        if (merge_flag[a] == c_hi - c_lo) {
-          if (row == 0) p.counters[2 * s.item + a] = 0;  // ready for the next launch
-          __threadfence();
-          auto part_of = [&](int c) -> const float* {
-            const int64_t clo = Sched::cta_lo(p, c);
-            const bool first = clo >= s.item_step0;   // the part starts the range of CTA c
-            return p.part + (static_cast<int64_t>(2 * c + (first ? 0 : 1)) * kPartFloats + a * kPartTileFloats);
-          };
-          float m_all = -INFINITY;
-          for (int c = c_lo; c <= c_hi; ++c) m_all = fmaxf(m_all, __ldcg(part_of(c) + 128 * 128 + row));
-          float l_all = 0.f;
-          for (int c = c_lo; c <= c_hi; ++c) {
-            const float* pc = part_of(c);
-            l_all += __ldcg(pc + 128 * 128 + 128 + row) *
-                     ex2((__ldcg(pc + 128 * 128 + row) - m_all) * p.scale_log2e);
-          }
+        const float l_all = l_run[a] + xc[(1 - half) * 128 + row];
+        const uint32_t t_O = t_lane + 256 + a * 128 + 64 * half;
+        const int n = (2 * s.qp + a) * kTileM + row;
+        uint4* dst = reinterpret_cast<uint4*>(
+            out + ((static_cast<int64_t>(s.b) * p.L + n) * p.Hn + s.h) * kHeadDim + 64 * half);
+        const bool whole = (s.t0 == 0 && s.t1 == s.tiles);
+        if (whole) {
+          // O / l -> bf16 -> out[b][n][h][64*half ...]
           const float inv_l = 1.f / l_all;
-#pragma unroll 1
-          for (int q = 0; q < 4; ++q) {
-            float acc[32];
 #pragma unroll
-            for (int i = 0; i < 32; ++i) acc[i] = 0.f;
-            for (int c = c_lo; c <= c_hi; ++c) {
-              const float* pc = part_of(c);
-              const float sc = ex2((__ldcg(pc + 128 * 128 + row) - m_all) * p.scale_log2e);
-#pragma unroll
-              for (int i = 0; i < 32; ++i) acc[i] = fmaf(__ldcg(pc + (q * 32 + i) * 128 + row), sc, acc[i]);
-            }
+          for (int q = 0; q < 2; ++q) {
+            uint32_t o[32];
+            tmem_ld32(t_O + q * 32, o);
+            tc_wait_ld();
             if (n < p.L) {
 #pragma unroll
               for (int i = 0; i < 4; ++i) {
                 uint4 vv;
-                vv.x = pack_bf16x2(acc[8 * i + 0] * inv_l, acc[8 * i + 1] * inv_l);
-                vv.y = pack_bf16x2(acc[8 * i + 2] * inv_l, acc[8 * i + 3] * inv_l);
-                vv.z = pack_bf16x2(acc[8 * i + 4] * inv_l, acc[8 * i + 5] * inv_l);
-                vv.w = pack_bf16x2(acc[8 * i + 6] * inv_l, acc[8 * i + 7] * inv_l);
+                vv.x = pack_bf16x2(__uint_as_float(o[8 * i + 0]) * inv_l, __uint_as_float(o[8 * i + 1]) * inv_l);
+                vv.y = pack_bf16x2(__uint_as_float(o[8 * i + 2]) * inv_l, __uint_as_float(o[8 * i + 3]) * inv_l);
+                vv.z = pack_bf16x2(__uint_as_float(o[8 * i + 4]) * inv_l, __uint_as_float(o[8 * i + 5]) * inv_l);
+                vv.w = pack_bf16x2(__uint_as_float(o[8 * i + 6]) * inv_l, __uint_as_float(o[8 * i + 7]) * inv_l);
                 dst[q * 4 + i] = vv;
               }
             }
           }
+        } else {
+          // part of a split item: publish (O, m, l), count the arrival; the last part to arrive
+          // merges all of them in part order (a fixed order, so the result does not depend on
+          // which CTA happens to be last)
+          float* mine = p.part + (static_cast<int64_t>(2 * blockIdx.x + (s.first_in_cta ? 0 : 1)) * kPartFloats +
+                                  a * kPartTileFloats);
+#pragma unroll
+          for (int q = 0; q < 2; ++q) {
+            uint32_t o[32];
+            tmem_ld32(t_O + q * 32, o);
+            tc_wait_ld();
+#pragma unroll
+            for (int i = 0; i < 32; ++i) mine[(64 * half + q * 32 + i) * 128 + row] = __uint_as_float(o[i]);
+          }
+          if (half == 0) {
+            mine[128 * 128 + row] = m_run[a];
+            mine[128 * 128 + 128 + row] = l_all;
+          }
+          __threadfence();
+          softmax_barrier();
+          const int c_lo = Sched::cta_of(p, s.item_step0);
+          const int c_hi = Sched::cta_of(p, s.item_step0 + s.tiles - 1);
+          if (tid == 0) *merge_flag = atomicAdd(p.counters + 2 * s.item + a, 1);
+          softmax_barrier();
+          const bool last = (*merge_flag == c_hi - c_lo);
+          softmax_barrier();  // everyone has read the flag before it can be written again
+          if (last) {
+            if (tid == 0) p.counters[2 * s.item + a] = 0;  // ready for the next launch
+            __threadfence();
+            auto part_of = [&](int c) -> const float* {
+              const int64_t clo = Sched::cta_lo(p, c);
+              const bool first = clo >= s.item_step0;   // the part starts the range of CTA c
+              return p.part + (static_cast<int64_t>(2 * c + (first ? 0 : 1)) * kPartFloats + a * kPartTileFloats);
+            };
+            float m_all = -INFINITY;
+            for (int c = c_lo; c <= c_hi; ++c) m_all = fmaxf(m_all, __ldcg(part_of(c) + 128 * 128 + row));
+            float l_sum = 0.f;
+            for (int c = c_lo; c <= c_hi; ++c) {
+              const float* pc = part_of(c);
+              l_sum += __ldcg(pc + 128 * 128 + 128 + row) *
+                       ex2((__ldcg(pc + 128 * 128 + row) - m_all) * p.scale_log2e);
+            }
+            const float inv_l = 1.f / l_sum;
+#pragma unroll 1
+            for (int q = 0; q < 2; ++q) {
+              float acc[32];
+#pragma unroll
+              for (int i = 0; i < 32; ++i) acc[i] = 0.f;
+              for (int c = c_lo; c <= c_hi; ++c) {
+                const float* pc = part_of(c);
+                const float sc = ex2((__ldcg(pc + 128 * 128 + row) - m_all) * p.scale_log2e);
+#pragma unroll
+                for (int i = 0; i < 32; ++i)
+                  acc[i] = fmaf(__ldcg(pc + (64 * half + q * 32 + i) * 128 + row), sc, acc[i]);
+              }
+              if (n < p.L) {
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                  uint4 vv;
+                  vv.x = pack_bf16x2(acc[8 * i + 0] * inv_l, acc[8 * i + 1] * inv_l);
+                  vv.y = pack_bf16x2(acc[8 * i + 2] * inv_l, acc[8 * i + 3] * inv_l);
+                  vv.z = pack_bf16x2(acc[8 * i + 4] * inv_l, acc[8 * i + 5] * inv_l);
+                  vv.w = pack_bf16x2(acc[8 * i + 6] * inv_l, acc[8 * i + 7] * inv_l);
+                  dst[q * 4 + i] = vv;
+                }
+              }
+            }
+          }
         }
+        tc_fence_before();
       }
-      tc_fence_before();
     }
   }
 
