@@ -68,12 +68,13 @@ struct AttnParams {
   int32_t n_streams;
   float scale_log2e;        // log2(e) / sqrt(128)
   int32_t items_per_stream; // Hn * q_pairs
-  int64_t total_steps;      // sum over items of their key tiles
+  int32_t full_rounds;      // whole rounds per stream: items_per_stream / gridDim.x
+  int64_t total_steps;      // remainder: sum over the leftover items of their key tiles
   float* part;              // workspace: partial results of split items, kPartFloats per slot
   int* counters;            // workspace: arrivals per (item, query tile), zero between launches
   int32_t first_frame[kMaxStreamsPerLaunch];  // first attended absolute frame of stream b
   int32_t n_frames[kMaxStreamsPerLaunch];     // attended frames of stream b
-  int64_t step_base[kMaxStreamsPerLaunch];    // steps of all streams before b
+  int64_t step_base[kMaxStreamsPerLaunch];    // remainder steps of all streams before b
 };
 
 // Partial result of one query tile of a split item: O[col][row] (unnormalised, relative to the
@@ -91,12 +92,19 @@ struct Seg {
   bool first_in_cta;  // this segment starts the CTA's range
 };
 
-// The (item, key tile) steps of the launch form one sequence, ordered stream, head, query
-// pair, key tile, and every CTA takes an equal contiguous share of it.  An item that straddles
-// a CTA boundary is split along its keys; the parts are merged by whichever CTA finishes last.
-// Neighbouring CTAs work on the same head, so its K/V is shared through L2.
+// Work split.  Items are ordered stream, head, query pair, so neighbouring CTAs work on the
+// same head and share its K/V through L2.
+//   1. Whole rounds: while a stream still has at least gridDim.x items, CTA c takes item
+//      (round * gridDim.x + c) whole.  All CTAs walk the key tiles in step, so a K/V tile is
+//      fetched from HBM once and then hit in L2 by the other CTAs of the head.
+//   2. Remainder: the leftover items of all streams (fewer than gridDim.x per stream) form one
+//      sequence of (item, key tile) steps, and every CTA takes an equal contiguous share of
+//      it.  An item that straddles a CTA boundary is split along its keys; the parts are
+//      merged by whichever CTA finishes last.  Only a few heads are live here, so their K/V
+//      stays in L2 although the CTAs are no longer in step.
 struct Sched {
   int64_t lo, hi, cur;
+  int b_round, round;   // position in the whole rounds
   const AttnParams& p;
   __device__ static int64_t cta_lo(const AttnParams& p, int64_t c) { return p.total_steps * c / gridDim.x; }
   __device__ static int cta_of(const AttnParams& p, int64_t step) {
@@ -109,24 +117,42 @@ struct Sched {
     lo = cta_lo(p, blockIdx.x);
     hi = cta_lo(p, blockIdx.x + 1);
     cur = lo;
+    b_round = 0;
+    round = 0;
+  }
+  __device__ void decode(Seg& s, int b, int in_stream) const {
+    s.b = b;
+    s.tiles = p.n_frames[b] * p.tiles_per_frame;
+    s.item = b * p.items_per_stream + in_stream;
+    s.qp = in_stream % p.q_pairs;
+    s.h = in_stream / p.q_pairs;
+    s.nq = (2 * s.qp + 1 < p.q_tiles) ? 2 : 1;
   }
   __device__ bool next(Seg& s) {
-    if (cur >= hi) return false;
+    while (b_round < p.n_streams) {          // whole rounds
+      if (round < p.full_rounds) {
+        decode(s, b_round, round * static_cast<int>(gridDim.x) + static_cast<int>(blockIdx.x));
+        s.t0 = 0;
+        s.t1 = s.tiles;
+        s.item_step0 = 0;
+        s.first_in_cta = false;
+        ++round;
+        return true;
+      }
+      round = 0;
+      ++b_round;
+    }
+    if (cur >= hi) return false;             // remainder
     int b = 0;
     while (b + 1 < p.n_streams && p.step_base[b + 1] <= cur) ++b;
     const int tiles = p.n_frames[b] * p.tiles_per_frame;
     const int64_t rel = cur - p.step_base[b];
-    const int in_stream = static_cast<int>(rel / tiles);
-    s.b = b;
-    s.tiles = tiles;
-    s.t0 = static_cast<int>(rel - static_cast<int64_t>(in_stream) * tiles);
+    const int left_item = static_cast<int>(rel / tiles);
+    decode(s, b, p.full_rounds * static_cast<int>(gridDim.x) + left_item);
+    s.t0 = static_cast<int>(rel - static_cast<int64_t>(left_item) * tiles);
     const int64_t left = hi - cur;
     s.t1 = (left < tiles - s.t0) ? s.t0 + static_cast<int>(left) : tiles;
-    s.item = b * p.items_per_stream + in_stream;
     s.item_step0 = cur - s.t0;
-    s.qp = in_stream % p.q_pairs;
-    s.h = in_stream / p.q_pairs;
-    s.nq = (2 * s.qp + 1 < p.q_tiles) ? 2 : 1;
     s.first_in_cta = (cur == lo);
     cur += s.t1 - s.t0;
     return true;
@@ -838,15 +864,21 @@ extern "C" int unstep_window_attn(const unstep_shape_t* shape, const int32_t* st
       p.first_frame[i] = lo;
       p.n_frames[i] = hi - lo;
     }
+    // grid: one CTA per SM, fewer when the whole launch is small
+    int64_t all_steps = 0;
+    for (int i = 0; i < nb; ++i)
+      all_steps += static_cast<int64_t>(p.items_per_stream) * p.n_frames[i] * p.tiles_per_frame;
+    int64_t want = all_steps / kMinStepsPerCta;
+    if (want < 1) want = 1;
+    const unsigned grid = static_cast<unsigned>(want < info.sm_count ? want : info.sm_count);
+    p.full_rounds = p.items_per_stream / static_cast<int>(grid);
+    const int leftover = p.items_per_stream - p.full_rounds * static_cast<int>(grid);
     int64_t steps = 0;
     for (int i = 0; i < nb; ++i) {
       p.step_base[i] = steps;
-      steps += static_cast<int64_t>(p.items_per_stream) * p.n_frames[i] * p.tiles_per_frame;
+      steps += static_cast<int64_t>(leftover) * p.n_frames[i] * p.tiles_per_frame;
     }
     p.total_steps = steps;
-    int64_t want = steps / kMinStepsPerCta;
-    if (want < 1) want = 1;
-    const unsigned grid = static_cast<unsigned>(want < info.sm_count ? want : info.sm_count);
     Workspace ws;
     if (!get_workspace(st, 2 * static_cast<size_t>(grid),
                        2 * static_cast<size_t>(nb) * p.items_per_stream, &ws))
