@@ -64,7 +64,7 @@ struct AttnParams {
   int32_t q_tiles;          // ceil(L / 128)
   int32_t q_pairs;          // ceil(q_tiles / 2)
   int32_t tiles_per_frame;  // ceil(T / 128)
-  int32_t tail_valid;       // valid keys in the last tile of a frame, 1..128
+  int32_t flat;             // 1: key tiles run across frame boundaries inside a slot run
   int32_t n_streams;
   float scale_log2e;        // log2(e) / sqrt(128)
   int32_t items_per_stream; // Hn * q_pairs
@@ -74,6 +74,11 @@ struct AttnParams {
   int* counters;            // workspace: arrivals per (item, query tile), zero between launches
   int32_t first_frame[kMaxStreamsPerLaunch];  // first attended absolute frame of stream b
   int32_t n_frames[kMaxStreamsPerLaunch];     // attended frames of stream b
+  int32_t tiles[kMaxStreamsPerLaunch];        // key tiles of one item of stream b
+  // flat mode: the window is at most two runs of consecutive ring slots (the ring wraps once);
+  // run A starts at ring row row0_a and has rows_a keys, run B starts at row 0 with rows_b keys
+  int32_t tiles_a[kMaxStreamsPerLaunch], row0_a[kMaxStreamsPerLaunch];
+  int32_t rows_a[kMaxStreamsPerLaunch], rows_b[kMaxStreamsPerLaunch];
   int64_t step_base[kMaxStreamsPerLaunch];    // remainder steps of all streams before b
 };
 
@@ -91,6 +96,42 @@ struct Seg {
   int64_t item_step0; // global step index of the item's first tile
   bool first_in_cta;  // this segment starts the CTA's range
 };
+
+// Where key tile j of an item of stream b lives and how many of its 128 keys are real.
+// Flat mode: tiles are cut from the runs of consecutive ring slots, so only the last tile of
+// a run is ragged; it is fetched through the per-frame map, whose zero fill ends it cleanly at
+// the end of its frame (a run ends on a frame end, and the ragged tile is shorter than a frame).
+// Per-frame mode (frames shorter than a tile): every tile lies inside one frame.
+struct TileInfo {
+  int valid;      // real keys in the tile, 1..128
+  bool framed;    // fetch through the (token, slot) map at (tok0, slot), else the flat map at row
+  int row, slot, tok0;
+};
+__device__ __forceinline__ TileInfo tile_info(const AttnParams& p, int b, int j) {
+  TileInfo t;
+  if (p.flat) {
+    const bool in_a = j < p.tiles_a[b];
+    const int tt = in_a ? j : j - p.tiles_a[b];
+    const int rows = in_a ? p.rows_a[b] : p.rows_b[b];
+    const int row0 = in_a ? p.row0_a[b] : 0;
+    const int ntl = in_a ? p.tiles_a[b] : p.tiles[b] - p.tiles_a[b];
+    const bool last = (tt == ntl - 1);
+    t.valid = last ? rows - kTileN * tt : kTileN;
+    t.framed = last;
+    t.row = row0 + kTileN * tt;
+    t.slot = (row0 + rows - 1) / p.T;
+    t.tok0 = p.T - t.valid;
+  } else {
+    const int fi = j / p.tiles_per_frame;
+    const int tt = j - fi * p.tiles_per_frame;
+    t.valid = (tt == p.tiles_per_frame - 1) ? p.T - kTileN * tt : kTileN;
+    t.framed = true;
+    t.row = 0;
+    t.slot = (p.first_frame[b] + fi) % p.C;
+    t.tok0 = kTileN * tt;
+  }
+  return t;
+}
 
 // Work split.  Items are ordered stream, head, query pair, so neighbouring CTAs work on the
 // same head and share its K/V through L2.
@@ -122,7 +163,7 @@ struct Sched {
   }
   __device__ void decode(Seg& s, int b, int in_stream) const {
     s.b = b;
-    s.tiles = p.n_frames[b] * p.tiles_per_frame;
+    s.tiles = p.tiles[b];
     s.item = b * p.items_per_stream + in_stream;
     s.qp = in_stream % p.q_pairs;
     s.h = in_stream / p.q_pairs;
@@ -145,7 +186,7 @@ struct Sched {
     if (cur >= hi) return false;             // remainder
     int b = 0;
     while (b + 1 < p.n_streams && p.step_base[b + 1] <= cur) ++b;
-    const int tiles = p.n_frames[b] * p.tiles_per_frame;
+    const int tiles = p.tiles[b];
     const int64_t rel = cur - p.step_base[b];
     const int left_item = static_cast<int>(rel / tiles);
     decode(s, b, p.full_rounds * static_cast<int>(gridDim.x) + left_item);
@@ -205,6 +246,32 @@ __device__ __forceinline__ void reg_alloc_200() { asm volatile("setmaxnreg.inc.s
 // P (bf16 pairs) overwrites the first 64 columns of S: this thread's 32 columns are written
 // only after the row's partner has loaded its scores (the barrier of the max exchange).
 // --------------------------------------------------------------------------------------
+// 2^x for a pair of floats without the MUFU pipe: x = n + f with n = round(x) (the add of
+// 1.5 * 2^23 leaves n in the low mantissa bits), 2^f by a cubic on [-0.5, 0.5] (relative error
+// 7.5e-5, far below the bf16 rounding of P), and n is added into the exponent field.
+// Inputs are clamped at -126 so that the exponent never wraps; -inf gives about 1e-38.
+__device__ __forceinline__ void exp2_poly_pair(uint64_t x2, float& p0, float& p1) {
+  float x0, x1;
+  unpack_f32x2(x2, x0, x1);
+  const uint64_t xc = pack_f32x2(fmaxf(x0, -126.f), fmaxf(x1, -126.f));
+  const uint64_t magic = pack_f32x2(12582912.f, 12582912.f);
+  const uint64_t t2 = add_f32x2(xc, magic);
+  const uint64_t n2 = add_f32x2(t2, pack_f32x2(-12582912.f, -12582912.f));
+  const uint64_t f2 = fma_f32x2(n2, pack_f32x2(-1.f, -1.f), xc);
+  uint64_t q2 = fma_f32x2(f2, pack_f32x2(0.055171650f, 0.055171650f), pack_f32x2(0.24261113f, 0.24261113f));
+  q2 = fma_f32x2(q2, f2, pack_f32x2(0.69326097f, 0.69326097f));
+  q2 = fma_f32x2(q2, f2, pack_f32x2(0.99992806f, 0.99992806f));
+  float q0, q1, t0, t1;
+  unpack_f32x2(q2, q0, q1);
+  unpack_f32x2(t2, t0, t1);
+  p0 = __uint_as_float(__float_as_uint(q0) + (__float_as_uint(t0) << 23));
+  p1 = __uint_as_float(__float_as_uint(q1) + (__float_as_uint(t1) << 23));
+}
+
+#ifndef UNSTEP_EMU_OF8
+#define UNSTEP_EMU_OF8 3   // of every 8 column pairs, this many take the polynomial instead of MUFU
+#endif
+
 __device__ __forceinline__ void softmax_barrier() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
 
 template <bool kMasked>
@@ -297,13 +364,16 @@ __device__ __forceinline__ bool softmax_tile(uint32_t t_S, uint32_t t_O, float c
   for (int i = 0; i < 32; ++i) {
     const uint64_t x2 = fma_f32x2(pack_f32x2(__uint_as_float(sreg[2 * i]), __uint_as_float(sreg[2 * i + 1])),
                                   c2, nm2);
-    float x0, x1;
-    unpack_f32x2(x2, x0, x1);
-#ifdef X_NOEXP
-    const float p0 = x0 * 1e-3f, p1 = x1 * 1e-3f;
-#else
-    const float p0 = ex2(x0), p1 = ex2(x1);
-#endif
+    float p0, p1;
+    if ((i & 7) < UNSTEP_EMU_OF8) {
+      // part of the exponentials runs on the FMA pipe: the MUFU pipe alone would bound the tile
+      exp2_poly_pair(x2, p0, p1);
+    } else {
+      float x0, x1;
+      unpack_f32x2(x2, x0, x1);
+      p0 = ex2(x0);
+      p1 = ex2(x1);
+    }
     acc[i & 3] = add_f32x2(acc[i & 3], pack_f32x2(p0, p1));
     preg[i] = pack_bf16x2(p0, p1);
   }
@@ -323,7 +393,8 @@ __device__ __forceinline__ bool softmax_tile(uint32_t t_S, uint32_t t_O, float c
 
 __global__ void __launch_bounds__(kThreads, 1)
 window_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
-                   const __grid_constant__ CUtensorMap tm_v, const AttnParams p,
+                   const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_kf,
+                   const __grid_constant__ CUtensorMap tm_vf, const AttnParams p,
                    __nv_bfloat16* __restrict__ out) {
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   const uint32_t smem_base = smem_u32(smem_raw);
@@ -377,7 +448,6 @@ window_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
   const Waiter w{abort_flag};
-  const int tail_n = (p.tail_valid + 15) & ~15;  // MMA N of the last tile of a frame
 
   if (warp >= 8) {
     reg_dealloc_96();
@@ -386,6 +456,8 @@ window_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
       prefetch_tensormap(&tm_q);
       prefetch_tensormap(&tm_k);
       prefetch_tensormap(&tm_v);
+      prefetch_tensormap(&tm_kf);
+      prefetch_tensormap(&tm_vf);
       Sched sched(p);
       Seg s;
       uint32_t kv_it = 0, q_it[2] = {0, 0};
@@ -401,33 +473,28 @@ window_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
           tma_load_4d(dst + kHalfBytes, &tm_q, bar, 64, s.h, n0, s.b);
           ++q_it[a];
         }
-        const int first_frame = p.first_frame[s.b];
-        int fi = s.t0 / p.tiles_per_frame;
-        int ti = s.t0 - fi * p.tiles_per_frame;
         for (int j = s.t0; j < s.t1 && ok; ++j) {
-          const int slot_f = (first_frame + fi) % p.C;
-          const int tok0 = ti * kTileN;
+          const TileInfo ti = tile_info(p, s.b, j);
           for (int kv = 0; kv < 2 && ok; ++kv) {
             const uint32_t st = kv_it % kStages;
             ok = w.wait(bar_kv_empty + 8 * st, ((kv_it / kStages) & 1) ^ 1);
             if (!ok) break;
             const uint32_t dst = sKV + st * kTileBytes, bar = bar_kv_full + 8 * st;
-            const CUtensorMap* tm = kv == 0 ? &tm_k : &tm_v;
 #if defined(X_NOTMA)
             mbar_arrive(bar);
-#elif defined(X_HALFTMA)
-            mbar_expect_tx(bar, kHalfBytes);
-            tma_load_5d(dst, tm, bar, 0, s.h, tok0, slot_f, s.b);
 #else
             mbar_expect_tx(bar, kTileBytes);
-            tma_load_5d(dst, tm, bar, 0, s.h, tok0, slot_f, s.b);
-            tma_load_5d(dst + kHalfBytes, tm, bar, 64, s.h, tok0, slot_f, s.b);
+            if (ti.framed) {
+              const CUtensorMap* tm = kv == 0 ? &tm_k : &tm_v;
+              tma_load_5d(dst, tm, bar, 0, s.h, ti.tok0, ti.slot, s.b);
+              tma_load_5d(dst + kHalfBytes, tm, bar, 64, s.h, ti.tok0, ti.slot, s.b);
+            } else {
+              const CUtensorMap* tm = kv == 0 ? &tm_kf : &tm_vf;
+              tma_load_4d(dst, tm, bar, 0, s.h, ti.row, s.b);
+              tma_load_4d(dst + kHalfBytes, tm, bar, 64, s.h, ti.row, s.b);
+            }
 #endif
             ++kv_it;
-          }
-          if (++ti == p.tiles_per_frame) {
-            ti = 0;
-            ++fi;
           }
         }
       }
@@ -443,8 +510,6 @@ window_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
       bool ok = true;
       const uint32_t idesc_pv = idesc_bf16_f32(kTileM, kHeadDim, 1);
       const uint32_t idesc_qk_full = idesc_bf16_f32(kTileM, kTileN, 0);
-      const uint32_t idesc_qk_tail = idesc_bf16_f32(kTileM, tail_n, 0);
-      const int k_steps_tail = tail_n >> 4;
       // descriptors are built once; per instruction only the start-address field moves
       const uint64_t dq = smem_desc_sw128(sQ + a * kTileBytes, 16, 1024);   // Q tile a, K-major
       const uint64_t dk0 = smem_desc_sw128(sKV, 16, 1024);                  // stage 0 as a K tile
@@ -452,9 +517,10 @@ window_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
       const uint32_t s_tmem = tmem_base + a * 128, o_tmem = tmem_base + 256 + a * 128;
       const uint32_t my_s_full = bar_s_full + 8 * a, my_p_half = bar_p_half + 16 * a;
 
-      auto issue_qk = [&](uint32_t stage, bool tail) {
+      // a ragged tile runs with N (for Q K^T) and K (for P V) rounded up to 16 keys
+      auto issue_qk = [&](uint32_t stage, int valid) {
         const uint64_t dk = dk0 + static_cast<uint64_t>((stage * kTileBytes) >> 4);
-        const uint32_t idesc = tail ? idesc_qk_tail : idesc_qk_full;
+        const uint32_t idesc = valid == kTileN ? idesc_qk_full : idesc_bf16_f32(kTileM, (valid + 15) & ~15, 0);
 #pragma unroll
         for (int k = 0; k < 8; ++k) {
           const uint64_t off = static_cast<uint64_t>(((k >> 2) * kHalfBytes + (k & 3) * 32) >> 4);
@@ -480,7 +546,7 @@ window_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
       while (ok && sched.next(s)) {
         const bool part = a < s.nq;   // a lone last query tile leaves warp 1 only the bookkeeping
         const int n = s.t1 - s.t0;
-        int ti = s.t0 % p.tiles_per_frame;  // tile index inside its frame
+        int valid = tile_info(p, s.b, s.t0).valid;  // real keys of the tile S is being computed for
         if (part) {
           ok = w.wait(bar_q_full + 8 * a, q_it & 1);
           if (!ok) break;
@@ -492,19 +558,19 @@ window_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         ++kv_it;
         if (part) {
           tc_fence_after();
-          issue_qk(kst, ti == p.tiles_per_frame - 1);
+          issue_qk(kst, valid);
         } else {
           mbar_arrive(bar_kv_empty + 8 * kst);
         }
         for (int j = 0; j < n; ++j) {
-          const int k_steps = (ti == p.tiles_per_frame - 1) ? k_steps_tail : 8;
-          if (++ti == p.tiles_per_frame) ti = 0;
+          const int k_steps = (valid + 15) >> 4;
           const uint32_t vst = kv_it % kStages;
           ok = w.wait(bar_kv_full + 8 * vst, (kv_it / kStages) & 1);
           if (!ok) break;
           ++kv_it;
           const bool more = j + 1 < n;
           if (more) {
+            valid = tile_info(p, s.b, s.t0 + j + 1).valid;
             kst = kv_it % kStages;
             ok = w.wait(bar_kv_full + 8 * kst, (kv_it / kStages) & 1);
             if (!ok) break;
@@ -525,7 +591,7 @@ window_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
             issue_pv_half(dv, 1, k_steps, true);
             tc_commit(bar_kv_empty + 8 * vst);
             TRACE(2 + a, sp_it, 4);
-            if (more) issue_qk(kst, ti == p.tiles_per_frame - 1);
+            if (more) issue_qk(kst, valid);
             TRACE(2 + a, sp_it, 5);
             ++sp_it;
           } else {
@@ -552,10 +618,9 @@ window_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
     bool ok = true;
     while (ok && sched.next(s)) {
       float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};
-      int ti = s.t0 % p.tiles_per_frame;
       for (int j = s.t0; j < s.t1 && ok; ++j) {
-        const bool tail = (ti == p.tiles_per_frame - 1) && p.tail_valid < kTileN;
-        if (++ti == p.tiles_per_frame) ti = 0;
+        const int valid = tile_info(p, s.b, j).valid;
+        const bool tail = valid < kTileN;
 #pragma unroll
         for (int a = 0; a < 2; ++a) {
           if (a >= s.nq) break;
@@ -567,7 +632,7 @@ window_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
           const uint32_t t_S = t_lane + a * 128, t_O = t_lane + 256 + a * 128;
           const uint32_t bar_p = bar_p_half + 16 * a + 8 * half;
           if (tail)
-            ok = softmax_tile<true>(t_S, t_O, p.scale_log2e, p.tail_valid, j == s.t0, half, row, xc,
+            ok = softmax_tile<true>(t_S, t_O, p.scale_log2e, valid, j == s.t0, half, row, xc,
                                     abort_flag, m_run[a], l_run[a], bar_p, a, it[a]);
           else
             ok = softmax_tile<false>(t_S, t_O, p.scale_log2e, kTileN, j == s.t0, half, row, xc,
@@ -851,7 +916,7 @@ extern "C" int unstep_window_attn(const unstep_shape_t* shape, const int32_t* st
   p.q_tiles = static_cast<int32_t>((L + kTileM - 1) / kTileM);
   p.q_pairs = (p.q_tiles + 1) / 2;
   p.tiles_per_frame = static_cast<int32_t>((T + kTileN - 1) / kTileN);
-  p.tail_valid = static_cast<int32_t>(T) - (p.tiles_per_frame - 1) * kTileN;
+  p.flat = (T >= kTileN) ? 1 : 0;  // a ragged tile must fit inside one frame
   p.scale_log2e = 1.4426950408889634f / sqrtf(static_cast<float>(kHeadDim));
   p.items_per_stream = p.Hn * p.q_pairs;
 
@@ -863,11 +928,23 @@ extern "C" int unstep_window_attn(const unstep_shape_t* shape, const int32_t* st
       const int lo = hi - window_frames > 0 ? hi - window_frames : 0;
       p.first_frame[i] = lo;
       p.n_frames[i] = hi - lo;
+      if (p.flat) {
+        const int slot0 = lo % shape->ring_frames;
+        const int frames_a = (hi - lo) < shape->ring_frames - slot0 ? (hi - lo) : shape->ring_frames - slot0;
+        p.row0_a[i] = slot0 * p.T;
+        p.rows_a[i] = frames_a * p.T;
+        p.rows_b[i] = (hi - lo - frames_a) * p.T;
+        p.tiles_a[i] = (p.rows_a[i] + kTileN - 1) / kTileN;
+        p.tiles[i] = p.tiles_a[i] + (p.rows_b[i] + kTileN - 1) / kTileN;
+      } else {
+        p.row0_a[i] = p.rows_a[i] = p.rows_b[i] = p.tiles_a[i] = 0;
+        p.tiles[i] = (hi - lo) * p.tiles_per_frame;
+      }
     }
     // grid: one CTA per SM, fewer when the whole launch is small
     int64_t all_steps = 0;
     for (int i = 0; i < nb; ++i)
-      all_steps += static_cast<int64_t>(p.items_per_stream) * p.n_frames[i] * p.tiles_per_frame;
+      all_steps += static_cast<int64_t>(p.items_per_stream) * p.tiles[i];
     int64_t want = all_steps / kMinStepsPerCta;
     if (want < 1) want = 1;
     const unsigned grid = static_cast<unsigned>(want < info.sm_count ? want : info.sm_count);
@@ -876,7 +953,7 @@ extern "C" int unstep_window_attn(const unstep_shape_t* shape, const int32_t* st
     int64_t steps = 0;
     for (int i = 0; i < nb; ++i) {
       p.step_base[i] = steps;
-      steps += static_cast<int64_t>(leftover) * p.n_frames[i] * p.tiles_per_frame;
+      steps += static_cast<int64_t>(leftover) * p.tiles[i];
     }
     p.total_steps = steps;
     Workspace ws;
@@ -890,15 +967,18 @@ extern "C" int unstep_window_attn(const unstep_shape_t* shape, const int32_t* st
     const char* vb = static_cast<const char*>(ring_v) + static_cast<uint64_t>(b0) * C * T * row_bytes;
     __nv_bfloat16* ob = reinterpret_cast<__nv_bfloat16*>(static_cast<char*>(out) +
                                                          static_cast<uint64_t>(b0) * L * row_bytes);
-    CUtensorMap tm_q, tm_k, tm_v;
+    CUtensorMap tm_q, tm_k, tm_v, tm_kf, tm_vf;
     const uint64_t qdims[4] = {kHeadDim, Hn, L, static_cast<uint64_t>(nb)};
     const uint64_t qstr[3] = {kHeadDim * 2, row_bytes, L * row_bytes};
     const uint64_t rdims[5] = {kHeadDim, Hn, T, C, static_cast<uint64_t>(nb)};
     const uint64_t rstr[4] = {kHeadDim * 2, row_bytes, T * row_bytes, C * T * row_bytes};
+    const uint64_t fdims[4] = {kHeadDim, Hn, C * T, static_cast<uint64_t>(nb)};   // ring rows, flat
+    const uint64_t fstr[3] = {kHeadDim * 2, row_bytes, C * T * row_bytes};
     if (!make_map(&tm_q, qb, 4, qdims, qstr, 2) || !make_map(&tm_k, kb, 5, rdims, rstr, 2) ||
-        !make_map(&tm_v, vb, 5, rdims, rstr, 2))
+        !make_map(&tm_v, vb, 5, rdims, rstr, 2) || !make_map(&tm_kf, kb, 4, fdims, fstr, 2) ||
+        !make_map(&tm_vf, vb, 4, fdims, fstr, 2))
       return UNSTEP_ERR_CUDA;
-    window_attn_kernel<<<grid, kThreads, kAttnSmemBytes, st>>>(tm_q, tm_k, tm_v, p, ob);
+    window_attn_kernel<<<grid, kThreads, kAttnSmemBytes, st>>>(tm_q, tm_k, tm_v, tm_kf, tm_vf, p, ob);
     g_launches.fetch_add(1);
     if (cudaGetLastError() != cudaSuccess) return UNSTEP_ERR_CUDA;
   }
