@@ -35,7 +35,7 @@ METRIC = "windowed-attn TFLOP/s at 1.3B-class shape (whole layer-chunk step: tab
 WORKLOAD = "cfg2"
 # dram__bytes_read.sum + dram__bytes_write.sum of one window_attn launch at this workload,
 # from the ncu capture summarised under profiles/ (None until captured)
-ATTN_DRAM_TRAFFIC_BYTES = None
+ATTN_DRAM_TRAFFIC_BYTES = 346_073_088
 
 
 def load_peaks():
@@ -164,15 +164,12 @@ def run_reference(args):
 # --------------------------------------------------------------------------- CUDA arm
 def run_ours(args):
     import torch
-    import torch.distributed as dist
     import paper_2609_32518_b200 as U
+    from paper_2609_32518_b200 import dist as D
 
-    rank = int(os.environ.get("RANK", "0"))
-    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank, local_rank, world = D.env_ranks()
     torch.cuda.set_device(local_rank)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    D.init("nccl", torch.device("cuda", local_rank))
 
     peaks = load_peaks()
     wl = W.WORKLOADS[WORKLOAD]
@@ -234,16 +231,10 @@ def run_ours(args):
         out_host.copy_(out.view(torch.int16), non_blocking=True)
 
     def barrier():
-        if world > 1:
-            dist.barrier()
-        torch.cuda.synchronize()
+        D.barrier(dev)
 
     def max_over_ranks(x: float) -> float:
-        if world == 1:
-            return x
-        t = torch.tensor([x], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item())
+        return D.max_over_ranks(x, dev)
 
     K, Wm = args.steps, max(args.warmup, 3)
     flops_step = wl.attn_flops(wf)
@@ -286,8 +277,7 @@ def run_ours(args):
     h2d = 3 * host_sets[0][0].numel() * 2
     d2h = out_host.numel() * 2
 
-    if world > 1:
-        dist.destroy_process_group()
+    D.finalize()
     if rank != 0:
         return
 
@@ -324,7 +314,7 @@ def run_ours(args):
     if not args.no_cpu_baseline and world == 1:
         cores = len(os.sched_getaffinity(0))
         oracle_sample(wl, 1, 256)
-        dt, fl, desc = oracle_sample(wl, 4, 2340)
+        dt, fl, desc = oracle_sample(wl, wl.shape.heads, wl.shape.chunk_tokens)
         line["cpu_baseline"] = {"value": fl / dt / 1e12, "unit": "TFLOP/s", "cores": cores, "kind": "oracle",
                                 "sample": desc, "seconds": dt}
     print(json.dumps(line))

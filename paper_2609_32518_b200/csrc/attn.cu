@@ -269,7 +269,7 @@ __device__ __forceinline__ void exp2_poly_pair(uint64_t x2, float& p0, float& p1
 }
 
 #ifndef UNSTEP_EMU_OF8
-#define UNSTEP_EMU_OF8 3   // of every 8 column pairs, this many take the polynomial instead of MUFU
+#define UNSTEP_EMU_OF8 2   // of every 8 column pairs, this many take the polynomial instead of MUFU
 #endif
 
 __device__ __forceinline__ void softmax_barrier() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
@@ -280,36 +280,10 @@ __device__ __forceinline__ bool softmax_tile(uint32_t t_S, uint32_t t_O, float c
                                              volatile int* abort_flag, float& m_run, float& l_run,
                                              uint32_t bar_p, int trace_role, int trace_tile) {
   uint32_t sreg[64];
-#ifdef X_NOLD
-#pragma unroll
-  for (int i = 0; i < 64; ++i) sreg[i] = 0x3f800000u + i + row;
-#else
   tmem_ld32(t_S + 64 * half, sreg);
   tmem_ld32(t_S + 64 * half + 32, sreg + 32);
   tc_wait_ld();
-#endif
   TRACE(trace_role, trace_tile, 2);
-#ifdef X_NOSOFTMAX
-  {
-    xchg[half * 128 + row] = 0.f;
-    softmax_barrier();
-    if (*abort_flag) return false;
-    uint32_t preg[32];
-#pragma unroll
-    for (int i = 0; i < 32; ++i) preg[i] = sreg[i] ^ sreg[i + 32];
-#ifndef X_NOLD
-    tmem_st32(t_S + 32 * half, preg);
-    tc_wait_st();
-#else
-    if (preg[0] == 0x12345u) l_run += 1.f;
-#endif
-    tc_fence_before();
-    mbar_arrive(bar_p);
-    l_run += 1.f;
-    m_run = 0.f;
-    return true;
-  }
-#endif
   if (kMasked) {
 #pragma unroll
     for (int i = 0; i < 64; ++i)
@@ -480,9 +454,6 @@ window_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
             ok = w.wait(bar_kv_empty + 8 * st, ((kv_it / kStages) & 1) ^ 1);
             if (!ok) break;
             const uint32_t dst = sKV + st * kTileBytes, bar = bar_kv_full + 8 * st;
-#if defined(X_NOTMA)
-            mbar_arrive(bar);
-#else
             mbar_expect_tx(bar, kTileBytes);
             if (ti.framed) {
               const CUtensorMap* tm = kv == 0 ? &tm_k : &tm_v;
@@ -493,7 +464,6 @@ window_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
               tma_load_4d(dst, tm, bar, 0, s.h, ti.row, s.b);
               tma_load_4d(dst + kHalfBytes, tm, bar, 64, s.h, ti.row, s.b);
             }
-#endif
             ++kv_it;
           }
         }
@@ -524,9 +494,7 @@ window_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
 #pragma unroll
         for (int k = 0; k < 8; ++k) {
           const uint64_t off = static_cast<uint64_t>(((k >> 2) * kHalfBytes + (k & 3) * 32) >> 4);
-#ifndef X_NOQK
           mma_ss(s_tmem, dq + off, dk + off, idesc, k > 0);
-#endif
         }
         tc_commit(my_s_full);
         tc_commit(bar_kv_empty + 8 * stage);
@@ -534,11 +502,7 @@ window_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
       auto issue_pv_half = [&](uint64_t dv, int half, int k_steps, bool accumulate) {
 #pragma unroll
         for (int k = 4 * half; k < 4 * half + 4; ++k)
-#ifndef X_NOPV
           if (k < k_steps)
-#else
-          if (k < k_steps && k == 100)
-#endif
             mma_ts(o_tmem, s_tmem + k * 8, dv + static_cast<uint64_t>((k * 2048) >> 4), idesc_pv,
                    (accumulate || k > 0) ? 1u : 0u);
       };
@@ -882,9 +846,14 @@ static void reset_workspace_counters() {
 
 using namespace unstep;
 
-extern "C" int unstep_window_attn(const unstep_shape_t* shape, const int32_t* start_frame,
-                                  int32_t window_frames, const void* q_rot, const void* ring_k,
-                                  const void* ring_v, void* out, void* cuda_stream) {
+// Hands out the scratch of one launch: `slots` partial-result slots and `n_counters` zeroed
+// arrival counters.
+typedef bool (*ScratchFn)(cudaStream_t st, size_t slots, size_t n_counters, Workspace* out);
+
+// Validation, work split, tensor maps and launch shared by the attention entry points.
+static int window_attn_run(const unstep_shape_t* shape, const int32_t* start_frame,
+                           int32_t window_frames, const void* q_rot, const void* ring_k,
+                           const void* ring_v, void* out, void* cuda_stream, ScratchFn scratch) {
   int rc = check_shape(shape, true);
   if (rc != UNSTEP_OK) return rc;
   const void* ptrs[] = {start_frame, q_rot, ring_k, ring_v, out};
@@ -957,8 +926,7 @@ extern "C" int unstep_window_attn(const unstep_shape_t* shape, const int32_t* st
     }
     p.total_steps = steps;
     Workspace ws;
-    if (!get_workspace(st, 2 * static_cast<size_t>(grid),
-                       2 * static_cast<size_t>(nb) * p.items_per_stream, &ws))
+    if (!scratch(st, 2 * static_cast<size_t>(grid), 2 * static_cast<size_t>(nb) * p.items_per_stream, &ws))
       return UNSTEP_ERR_CUDA;
     p.part = ws.part;
     p.counters = ws.counters;
@@ -992,6 +960,13 @@ extern "C" int unstep_debug_read_trace(long long* host_out) {
              ? UNSTEP_OK : UNSTEP_ERR_CUDA;
 }
 #endif
+
+extern "C" int unstep_window_attn(const unstep_shape_t* shape, const int32_t* start_frame,
+                                  int32_t window_frames, const void* q_rot, const void* ring_k,
+                                  const void* ring_v, void* out, void* cuda_stream) {
+  return window_attn_run(shape, start_frame, window_frames, q_rot, ring_k, ring_v, out, cuda_stream,
+                         get_workspace);
+}
 
 extern "C" int unstep_poll_status(void) {
   if (cudaDeviceSynchronize() != cudaSuccess) return UNSTEP_ERR_CUDA;
