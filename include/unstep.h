@@ -12,7 +12,8 @@
  * Conventions
  *   - Every tensor pointer is a DEVICE pointer unless the comment says HOST.
  *   - bf16 tensors are dense, row-major, 16-byte aligned; the caller owns all of
- *     them.  The library allocates no device memory.
+ *     them.  The only device memory the library creates is the scratch of
+ *     unstep_window_attn (one buffer per stream, made on first use and kept).
  *   - All work is enqueued on `cuda_stream` (a cudaStream_t passed as void*; NULL
  *     is the legacy default stream).  No call synchronises or reads device data.
  *   - Return value: 0 on success, a negative unstep_status otherwise.  Arguments
@@ -38,7 +39,8 @@ typedef enum {
   UNSTEP_ERR_INVALID_ARG = -1, /* null or misaligned pointer, bad size, bad window */
   UNSTEP_ERR_UNSUPPORTED = -2, /* head_dim != 128, device is not sm_100 */
   UNSTEP_ERR_CUDA = -3,        /* a CUDA runtime/driver call failed */
-  UNSTEP_ERR_TIMEOUT = -4      /* a bounded device-side wait expired (see unstep_poll_status) */
+  UNSTEP_ERR_TIMEOUT = -4,     /* a bounded device-side wait expired (see unstep_poll_status) */
+  UNSTEP_ERR_TOO_LARGE = -5    /* the problem does not fit the fixed scratch of a no-allocation call */
 } unstep_status;
 
 typedef struct {
@@ -118,6 +120,38 @@ int unstep_rope_kv_append(const unstep_shape_t* shape, const int32_t* start_fram
 int unstep_window_attn(const unstep_shape_t* shape, const int32_t* start_frame,
                        int32_t window_frames, const void* q_rot, const void* ring_k,
                        const void* ring_v, void* out, void* cuda_stream);
+
+/*
+ * unstep_window_attn for callers that must not allocate.  (The paper has no counterpart:
+ * this is a deployment variant of the call above, same arguments, same result.)
+ *
+ * unstep_window_attn keeps a scratch buffer per stream and creates it with cudaMalloc the first
+ * time it is needed.  That is not acceptable everywhere: a serving process whose device memory
+ * has been handed over in full to a framework's caching allocator has nothing left for a raw
+ * cudaMalloc to return; a latency-critical loop cannot take the device-wide synchronisation an
+ * allocation may imply; and some deployments forbid any allocation after start-up so that the
+ * memory footprint is known before the first request.  This entry point calls no cudaMalloc,
+ * cudaFree or any other allocating routine.  Its scratch is a fixed array that is part of the
+ * library image: about 39.8 MB of device memory on every GPU that loads the library, held
+ * until the process exits, whether or not this call is ever used.
+ *
+ * Limits (beyond them the call returns UNSTEP_ERR_TOO_LARGE and launches nothing):
+ *   - at most 148 SMs on the device (the array has two partial-result slots per SM);
+ *   - min(batch, 32) * heads * ceil(ceil(L / 128) / 2) <= 32768 (one pair of arrival counters
+ *     per work item of a launch).
+ *
+ * Set-up: the first call on each device looks up the device address of the array, with that
+ * device current, and remembers it.  Make that first call outside any stream capture.
+ *
+ * Sharing: every call on a device uses the same array, and the array keeps whatever the last
+ * call left in it.  Each call clears the counters it needs (stream-ordered, on cuda_stream)
+ * before its kernel runs.  Calls that can overlap on the GPU (different streams, or several
+ * host threads) race on the array and corrupt each other's results: serialise them, or use
+ * unstep_window_attn, which keeps one scratch per stream.
+ */
+int unstep_window_attn_noalloc(const unstep_shape_t* shape, const int32_t* start_frame,
+                               int32_t window_frames, const void* q_rot, const void* ring_k,
+                               const void* ring_v, void* out, void* cuda_stream);
 
 /* Static, human-readable text for a status code. */
 const char* unstep_strerror(int code);

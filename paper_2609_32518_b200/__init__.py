@@ -11,6 +11,7 @@ from .binding import (  # noqa: F401
     rope_table,
     rope_kv_append,
     window_attn,
+    window_attn_noalloc,
     poll_status,
     launch_count,
     strerror,

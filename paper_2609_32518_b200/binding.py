@@ -7,8 +7,8 @@ from ctypes import c_char_p, c_double, c_int, c_int32, c_int64, c_void_p, POINTE
 
 from . import build as _build
 
-EXPORTS = ("unstep_rope_table", "unstep_rope_kv_append", "unstep_window_attn", "unstep_strerror",
-           "unstep_poll_status", "unstep_launch_count")
+EXPORTS = ("unstep_rope_table", "unstep_rope_kv_append", "unstep_window_attn",
+           "unstep_window_attn_noalloc", "unstep_strerror", "unstep_poll_status", "unstep_launch_count")
 
 
 class UnstepError(RuntimeError):
@@ -57,6 +57,8 @@ def lib() -> ctypes.CDLL:
         L.unstep_window_attn.restype = c_int
         L.unstep_window_attn.argtypes = [POINTER(Shape), POINTER(c_int32), c_int32, c_void_p,
                                          c_void_p, c_void_p, c_void_p, c_void_p]
+        L.unstep_window_attn_noalloc.restype = c_int
+        L.unstep_window_attn_noalloc.argtypes = L.unstep_window_attn.argtypes
         L.unstep_strerror.restype = c_char_p
         L.unstep_strerror.argtypes = [c_int]
         L.unstep_poll_status.restype = c_int
@@ -139,6 +141,24 @@ def window_attn(shape: Shape, start_frame, window_frames: int, q_rot, ring_k, ri
         _dev_ptr(q_rot, bf, n, "q_rot"), _dev_ptr(ring_k, bf, nr, "ring_k"),
         _dev_ptr(ring_v, bf, nr, "ring_v"), _dev_ptr(out, bf, n, "out"), _stream_ptr(stream)),
         "unstep_window_attn")
+
+
+def window_attn_noalloc(shape: Shape, start_frame, window_frames: int, q_rot, ring_k, ring_v, out,
+                        stream=None):
+    """unstep_window_attn_noalloc: the same attention for callers that must not allocate device
+    memory (a process whose memory is owned by a framework allocator, a latency-critical loop,
+    a deployment with a fixed footprint).  Its scratch is a fixed ~40 MB array inside the
+    library; all calls on a device share it, so calls that may overlap on the GPU must be
+    serialised by the caller.  Raises UnstepError(-5) when the problem exceeds the array."""
+    import torch
+    bf = torch.bfloat16
+    n = shape.batch * shape.chunk_tokens * shape.heads * shape.head_dim
+    nr = shape.batch * shape.ring_frames * shape.tokens_per_frame * shape.heads * shape.head_dim
+    _check(lib().unstep_window_attn_noalloc(
+        ctypes.byref(shape), _starts(shape, start_frame), int(window_frames),
+        _dev_ptr(q_rot, bf, n, "q_rot"), _dev_ptr(ring_k, bf, nr, "ring_k"),
+        _dev_ptr(ring_v, bf, nr, "ring_v"), _dev_ptr(out, bf, n, "out"), _stream_ptr(stream)),
+        "unstep_window_attn_noalloc")
 
 
 def poll_status() -> int:

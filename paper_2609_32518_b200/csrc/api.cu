@@ -12,6 +12,7 @@ extern "C" const char* unstep_strerror(int code) {
     case UNSTEP_ERR_UNSUPPORTED: return "unsupported (head_dim must be 128, device must be sm_100)";
     case UNSTEP_ERR_CUDA: return "a CUDA call failed";
     case UNSTEP_ERR_TIMEOUT: return "a bounded device-side wait expired";
+    case UNSTEP_ERR_TOO_LARGE: return "too large for the fixed scratch of the no-allocation entry point";
     default: return "unknown status";
   }
 }

@@ -968,6 +968,74 @@ extern "C" int unstep_window_attn(const unstep_shape_t* shape, const int32_t* st
                          get_workspace);
 }
 
+// --------------------------------------------------------------------------
+// Attention without any allocation: the scratch is a fixed array in the library image.
+// --------------------------------------------------------------------------
+namespace unstep {
+
+constexpr int kStaticMaxCtas = 148;                      // two partial-result slots per CTA
+constexpr int kStaticMaxCounters = 2 * 32768;            // a pair of counters per work item
+constexpr size_t kStaticCounterBytes = sizeof(int) * kStaticMaxCounters;
+constexpr size_t kStaticScratchBytes =
+    kStaticCounterBytes + sizeof(float) * 2 * kStaticMaxCtas * static_cast<size_t>(kPartFloats);
+
+// Counters first, partial results after them.  In host code this name is only a handle for
+// cudaGetSymbolAddress: it is not a device address and must never be passed to a kernel.
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+
+constexpr int kMaxDevices = 64;
+static std::mutex g_static_mutex;
+static unsigned char* g_static_addr[kMaxDevices] = {};
+
+// Device address of the array on the current device (looked up once per device).
+static unsigned char* static_scratch_base() {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return nullptr;
+  std::lock_guard<std::mutex> lock(g_static_mutex);
+  if (g_static_addr[dev] == nullptr) {
+    void* ptr = nullptr;
+    if (cudaGetSymbolAddress(&ptr, g_static_scratch) != cudaSuccess || ptr == nullptr) return nullptr;
+    g_static_addr[dev] = static_cast<unsigned char*>(ptr);
+  }
+  return g_static_addr[dev];
+}
+
+// Scratch source of the no-allocation entry point: carve the fixed array, clear the counters
+// this launch will use (the array keeps the previous call's contents).
+static bool static_scratch(cudaStream_t st, size_t slots, size_t n_counters, Workspace* out) {
+  if (slots > 2 * static_cast<size_t>(kStaticMaxCtas) || n_counters > static_cast<size_t>(kStaticMaxCounters))
+    return false;
+  unsigned char* base = static_scratch_base();
+  if (base == nullptr) return false;
+  if (cudaMemsetAsync(base, 0, n_counters * sizeof(int), st) != cudaSuccess) return false;
+  out->counters = reinterpret_cast<int*>(base);
+  out->part = reinterpret_cast<float*>(base + kStaticCounterBytes);
+  out->slots = slots;
+  out->n_counters = n_counters;
+  return true;
+}
+
+}  // namespace unstep
+
+extern "C" int unstep_window_attn_noalloc(const unstep_shape_t* shape, const int32_t* start_frame,
+                                          int32_t window_frames, const void* q_rot, const void* ring_k,
+                                          const void* ring_v, void* out, void* cuda_stream) {
+  // size limits of the fixed array first, so that an oversized problem gets its own clear answer
+  int rc = check_shape(shape, true);
+  if (rc != UNSTEP_OK) return rc;
+  const int64_t L = static_cast<int64_t>(shape->grid_h) * shape->grid_w * shape->chunk_frames;
+  const int64_t q_pairs = ((L + kTileM - 1) / kTileM + 1) / 2;
+  const int64_t streams = shape->batch < kMaxStreamsPerLaunch ? shape->batch : kMaxStreamsPerLaunch;
+  if (2 * streams * shape->heads * q_pairs > kStaticMaxCounters) return UNSTEP_ERR_TOO_LARGE;
+  rc = check_device();
+  if (rc != UNSTEP_OK) return rc;
+  const DeviceInfo& info = device_info();
+  if (!info.ok) return UNSTEP_ERR_CUDA;
+  if (info.sm_count > kStaticMaxCtas) return UNSTEP_ERR_TOO_LARGE;
+  return window_attn_run(shape, start_frame, window_frames, q_rot, ring_k, ring_v, out, cuda_stream,
+                         static_scratch);
+}
+
 extern "C" int unstep_poll_status(void) {
   if (cudaDeviceSynchronize() != cudaSuccess) return UNSTEP_ERR_CUDA;
   int st = 0, zero = 0;
