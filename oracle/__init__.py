@@ -28,4 +28,10 @@ from .unstep_oracle import (  # noqa: F401
     explicit_window_attn,
     bf16_bits_to_f32,
     f32_to_bf16_bits_rne,
+    sink_slot,
+    sink_window_frames,
+    SinkRingState,
+    rope_kv_append_sink,
+    window_attn_sink,
+    explicit_frames_attn,
 )

@@ -307,3 +307,98 @@ def explicit_window_attn(history: ExplicitHistory, start_frame: int, chunk_frame
         v = bf16_bits_to_f32(v_bits[:, h]).astype(np.float64)
         out[:, hi_] = attention_rows(q, k, v)
     return out
+
+
+# ---------------------------------------------------------------------------
+# Sink + sliding window (Sec. "Limited KV attention window", appendix "KV attention
+# window"): the first `sink` latent frames are never evicted, the ring keeps the most
+# recent frames; once the cache is full a chunk attends the sink frames plus the
+# `recent` most recent frames, the current chunk included.  Before that (the recent
+# part still reaches back to the sink) it attends every frame so far.
+# ---------------------------------------------------------------------------
+
+def sink_slot(frame: int, sink_frames: int, ring_frames: int) -> int:
+    """Cache slot of an absolute frame: sink frames sit in a prefix that is never
+    overwritten, later frames in a ring behind it."""
+    if frame < sink_frames:
+        return frame
+    return sink_frames + (frame - sink_frames) % ring_frames
+
+
+def sink_window_frames(start_frame: int, chunk_frames: int, recent_frames: int, sink_attend: int):
+    """Absolute frames attended, in increasing order."""
+    hi = start_frame + chunk_frames
+    lo = max(0, hi - recent_frames)
+    return list(range(0, min(sink_attend, lo))) + list(range(lo, hi))
+
+
+@dataclass
+class SinkRingState:
+    """Per-layer KV cache with a sink prefix: bf16 bits [B, sink + C, T, Hn, 128]."""
+    batch: int
+    sink_frames: int
+    ring_frames: int
+    tokens_per_frame: int
+    heads: int
+    cache_k: np.ndarray = field(init=False)
+    cache_v: np.ndarray = field(init=False)
+
+    def __post_init__(self):
+        shape = (self.batch, self.sink_frames + self.ring_frames, self.tokens_per_frame, self.heads,
+                 HEAD_DIM)
+        self.cache_k = np.full(shape, SENTINEL, dtype=np.uint16)
+        self.cache_v = np.full(shape, SENTINEL, dtype=np.uint16)
+
+
+def rope_kv_append_sink(state: SinkRingState, start_frames, q_bits, k_bits, v_bits, cos, sin):
+    """R3 + R4 with the sink prefix: same rotation, slot = sink_slot(frame)."""
+    B, L, Hn, D = q_bits.shape
+    T = state.tokens_per_frame
+    assert D == HEAD_DIM and L % T == 0 and B == state.batch and Hn == state.heads
+    q_out = rope_rotate(q_bits, cos, sin)
+    k_rot = rope_rotate(k_bits, cos, sin)
+    for b in range(B):
+        s = int(start_frames[b])
+        for f in range(L // T):
+            slot = sink_slot(s + f, state.sink_frames, state.ring_frames)
+            state.cache_k[b, slot] = k_rot[b, f * T:(f + 1) * T]
+            state.cache_v[b, slot] = v_bits[b, f * T:(f + 1) * T]
+    return q_out
+
+
+def window_attn_sink(state: SinkRingState, start_frames, recent_frames: int, sink_attend: int,
+                     q_rot_bits: np.ndarray, chunk_frames: int, rows=None, heads=None) -> np.ndarray:
+    """A1 + A2 with the key set sink ∪ recent, read through sink_slot."""
+    B, L, Hn, D = q_rot_bits.shape
+    assert sink_attend <= state.sink_frames
+    rows = np.arange(L) if rows is None else np.asarray(rows, dtype=np.int64)
+    heads = list(range(Hn)) if heads is None else list(heads)
+    out = np.empty((B, len(rows), len(heads), D), dtype=np.float64)
+    for b in range(B):
+        frames = sink_window_frames(int(start_frames[b]), chunk_frames, recent_frames, sink_attend)
+        slots = [sink_slot(p, state.sink_frames, state.ring_frames) for p in frames]
+        k_bits = np.concatenate([state.cache_k[b, s] for s in slots], axis=0)
+        v_bits = np.concatenate([state.cache_v[b, s] for s in slots], axis=0)
+        for hi_, h in enumerate(heads):
+            q = bf16_bits_to_f32(q_rot_bits[b, rows, h]).astype(np.float64)
+            k = bf16_bits_to_f32(k_bits[:, h]).astype(np.float64)
+            v = bf16_bits_to_f32(v_bits[:, h]).astype(np.float64)
+            out[b, :, hi_] = attention_rows(q, k, v)
+    return out
+
+
+def explicit_frames_attn(history: ExplicitHistory, frames, q_rot_bits: np.ndarray, rows=None,
+                         heads=None) -> np.ndarray:
+    """Attention of q_rot_bits [L, Hn, 128] over an explicit list of frames of the history."""
+    L, Hn, D = q_rot_bits.shape
+    rows = np.arange(L) if rows is None else np.asarray(rows, dtype=np.int64)
+    heads = list(range(Hn)) if heads is None else list(heads)
+    k_bits = np.concatenate([history.k[p] for p in frames], axis=0)
+    v_bits = np.concatenate([history.v[p] for p in frames], axis=0)
+    out = np.empty((len(rows), len(heads), D), dtype=np.float64)
+    for hi_, h in enumerate(heads):
+        q = bf16_bits_to_f32(q_rot_bits[rows, h]).astype(np.float64)
+        k = bf16_bits_to_f32(k_bits[:, h]).astype(np.float64)
+        v = bf16_bits_to_f32(v_bits[:, h]).astype(np.float64)
+        out[:, hi_] = attention_rows(q, k, v)
+    return out
