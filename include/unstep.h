@@ -122,6 +122,34 @@ int unstep_window_attn(const unstep_shape_t* shape, const int32_t* start_frame,
                        const void* ring_v, void* out, void* cuda_stream);
 
 /*
+ * Sink + sliding window (Sec. "Limited KV attention window", appendix "KV attention window":
+ * the first 3 latent frames are kept as sink frames and never evicted, the 6 most recent
+ * frames, the current chunk included, form the sliding window; selected layers attend 2 sink
+ * frames and the same 6 recent frames).
+ *
+ * The cache of a stream has sink_frames slots in front of the ring:
+ *     cache_k, cache_v : bf16 [B, sink_frames + C, T, Hn, 128]
+ *     frame p lives in slot p                              if p <  sink_frames
+ *                      slot sink_frames + (p - sink_frames) mod C   otherwise.
+ * unstep_rope_kv_append_sink is unstep_rope_kv_append with that slot rule.
+ * unstep_window_attn_sink attends, for stream b with hi = start_frame[b] + Fc and
+ * lo = max(0, hi - recent_frames), the frames [0, min(sink_attend, lo)) and [lo, hi): while the
+ * recent part still reaches the sink this is every frame so far, afterwards sink + recent.
+ *   sink_frames  : >= 0; 0 makes both calls identical to the plain ones.
+ *   recent_frames: Fc <= recent_frames <= C.     sink_attend: 0 <= sink_attend <= sink_frames.
+ * All other arguments as in unstep_rope_kv_append / unstep_window_attn.
+ */
+int unstep_rope_kv_append_sink(const unstep_shape_t* shape, int32_t sink_frames,
+                               const int32_t* start_frame, const void* q_in, const void* k_in,
+                               const void* v_in, const float* cos, const float* sin,
+                               int64_t table_stream_stride, void* q_out, void* cache_k, void* cache_v,
+                               void* cuda_stream);
+int unstep_window_attn_sink(const unstep_shape_t* shape, int32_t sink_frames,
+                            const int32_t* start_frame, int32_t recent_frames, int32_t sink_attend,
+                            const void* q_rot, const void* cache_k, const void* cache_v, void* out,
+                            void* cuda_stream);
+
+/*
  * unstep_window_attn for callers that must not allocate.  (The paper has no counterpart:
  * this is a deployment variant of the call above, same arguments, same result.)
  *

@@ -12,6 +12,8 @@ from .binding import (  # noqa: F401
     rope_kv_append,
     window_attn,
     window_attn_noalloc,
+    rope_kv_append_sink,
+    window_attn_sink,
     poll_status,
     launch_count,
     strerror,

@@ -8,7 +8,8 @@ from ctypes import c_char_p, c_double, c_int, c_int32, c_int64, c_void_p, POINTE
 from . import build as _build
 
 EXPORTS = ("unstep_rope_table", "unstep_rope_kv_append", "unstep_window_attn",
-           "unstep_window_attn_noalloc", "unstep_strerror", "unstep_poll_status", "unstep_launch_count")
+           "unstep_window_attn_noalloc", "unstep_rope_kv_append_sink", "unstep_window_attn_sink",
+           "unstep_strerror", "unstep_poll_status", "unstep_launch_count")
 
 
 class UnstepError(RuntimeError):
@@ -59,6 +60,13 @@ def lib() -> ctypes.CDLL:
                                          c_void_p, c_void_p, c_void_p, c_void_p]
         L.unstep_window_attn_noalloc.restype = c_int
         L.unstep_window_attn_noalloc.argtypes = L.unstep_window_attn.argtypes
+        L.unstep_rope_kv_append_sink.restype = c_int
+        L.unstep_rope_kv_append_sink.argtypes = [POINTER(Shape), c_int32, POINTER(c_int32), c_void_p,
+                                                 c_void_p, c_void_p, c_void_p, c_void_p, c_int64,
+                                                 c_void_p, c_void_p, c_void_p, c_void_p]
+        L.unstep_window_attn_sink.restype = c_int
+        L.unstep_window_attn_sink.argtypes = [POINTER(Shape), c_int32, POINTER(c_int32), c_int32, c_int32,
+                                              c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]
         L.unstep_strerror.restype = c_char_p
         L.unstep_strerror.argtypes = [c_int]
         L.unstep_poll_status.restype = c_int
@@ -159,6 +167,38 @@ def window_attn_noalloc(shape: Shape, start_frame, window_frames: int, q_rot, ri
         _dev_ptr(q_rot, bf, n, "q_rot"), _dev_ptr(ring_k, bf, nr, "ring_k"),
         _dev_ptr(ring_v, bf, nr, "ring_v"), _dev_ptr(out, bf, n, "out"), _stream_ptr(stream)),
         "unstep_window_attn_noalloc")
+
+
+def rope_kv_append_sink(shape: Shape, sink_frames: int, start_frame, q_in, k_in, v_in, cos, sin, q_out,
+                        cache_k, cache_v, table_stream_stride: int = 0, stream=None):
+    """unstep_rope_kv_append_sink: the append with a sink prefix of `sink_frames` slots."""
+    import torch
+    bf = torch.bfloat16
+    n = shape.batch * shape.chunk_tokens * shape.heads * shape.head_dim
+    nr = (shape.batch * (shape.ring_frames + int(sink_frames)) * shape.tokens_per_frame * shape.heads
+          * shape.head_dim)
+    ntab = shape.chunk_tokens * 64 + (shape.batch - 1) * int(table_stream_stride)
+    _check(lib().unstep_rope_kv_append_sink(
+        ctypes.byref(shape), int(sink_frames), _starts(shape, start_frame),
+        _dev_ptr(q_in, bf, n, "q_in"), _dev_ptr(k_in, bf, n, "k_in"), _dev_ptr(v_in, bf, n, "v_in"),
+        _dev_ptr(cos, torch.float32, ntab, "cos"), _dev_ptr(sin, torch.float32, ntab, "sin"),
+        int(table_stream_stride), _dev_ptr(q_out, bf, n, "q_out"), _dev_ptr(cache_k, bf, nr, "cache_k"),
+        _dev_ptr(cache_v, bf, nr, "cache_v"), _stream_ptr(stream)), "unstep_rope_kv_append_sink")
+
+
+def window_attn_sink(shape: Shape, sink_frames: int, start_frame, recent_frames: int, sink_attend: int,
+                     q_rot, cache_k, cache_v, out, stream=None):
+    """unstep_window_attn_sink: attention over sink frames + the recent window."""
+    import torch
+    bf = torch.bfloat16
+    n = shape.batch * shape.chunk_tokens * shape.heads * shape.head_dim
+    nr = (shape.batch * (shape.ring_frames + int(sink_frames)) * shape.tokens_per_frame * shape.heads
+          * shape.head_dim)
+    _check(lib().unstep_window_attn_sink(
+        ctypes.byref(shape), int(sink_frames), _starts(shape, start_frame), int(recent_frames),
+        int(sink_attend), _dev_ptr(q_rot, bf, n, "q_rot"), _dev_ptr(cache_k, bf, nr, "cache_k"),
+        _dev_ptr(cache_v, bf, nr, "cache_v"), _dev_ptr(out, bf, n, "out"), _stream_ptr(stream)),
+        "unstep_window_attn_sink")
 
 
 def poll_status() -> int:

@@ -72,13 +72,16 @@ struct AttnParams {
   int64_t total_steps;      // remainder: sum over the leftover items of their key tiles
   float* part;              // workspace: partial results of split items, kPartFloats per slot
   int* counters;            // workspace: arrivals per (item, query tile), zero between launches
-  int32_t first_frame[kMaxStreamsPerLaunch];  // first attended absolute frame of stream b
-  int32_t n_frames[kMaxStreamsPerLaunch];     // attended frames of stream b
+  int32_t sink;             // S: cache slots [0, S) hold frames [0, S) for good, the ring follows
+  int32_t first_frame[kMaxStreamsPerLaunch];  // first frame of the recent part of stream b
+  int32_t n_sink[kMaxStreamsPerLaunch];       // sink frames attended in front of the recent part
   int32_t tiles[kMaxStreamsPerLaunch];        // key tiles of one item of stream b
-  // flat mode: the window is at most two runs of consecutive ring slots (the ring wraps once);
-  // run A starts at ring row row0_a and has rows_a keys, run B starts at row 0 with rows_b keys
-  int32_t tiles_a[kMaxStreamsPerLaunch], row0_a[kMaxStreamsPerLaunch];
-  int32_t rows_a[kMaxStreamsPerLaunch], rows_b[kMaxStreamsPerLaunch];
+  // flat mode: the attended frames are at most three runs of consecutive cache slots (sink
+  // prefix, ring up to its end, ring from its start); run r starts at cache row run_row0 and
+  // has run_rows keys, its tiles are [run_tile_end[r-1], run_tile_end[r])
+  int32_t run_row0[kMaxStreamsPerLaunch][3];
+  int32_t run_rows[kMaxStreamsPerLaunch][3];
+  int32_t run_tile_end[kMaxStreamsPerLaunch][3];
   int64_t step_base[kMaxStreamsPerLaunch];    // remainder steps of all streams before b
 };
 
@@ -110,11 +113,13 @@ struct TileInfo {
 __device__ __forceinline__ TileInfo tile_info(const AttnParams& p, int b, int j) {
   TileInfo t;
   if (p.flat) {
-    const bool in_a = j < p.tiles_a[b];
-    const int tt = in_a ? j : j - p.tiles_a[b];
-    const int rows = in_a ? p.rows_a[b] : p.rows_b[b];
-    const int row0 = in_a ? p.row0_a[b] : 0;
-    const int ntl = in_a ? p.tiles_a[b] : p.tiles[b] - p.tiles_a[b];
+    int r = 0;
+    if (j >= p.run_tile_end[b][0]) r = (j >= p.run_tile_end[b][1]) ? 2 : 1;
+    const int t_begin = r == 0 ? 0 : p.run_tile_end[b][r - 1];
+    const int tt = j - t_begin;
+    const int rows = p.run_rows[b][r];
+    const int row0 = p.run_row0[b][r];
+    const int ntl = p.run_tile_end[b][r] - t_begin;
     const bool last = (tt == ntl - 1);
     t.valid = last ? rows - kTileN * tt : kTileN;
     t.framed = last;
@@ -127,7 +132,9 @@ __device__ __forceinline__ TileInfo tile_info(const AttnParams& p, int b, int j)
     t.valid = (tt == p.tiles_per_frame - 1) ? p.T - kTileN * tt : kTileN;
     t.framed = true;
     t.row = 0;
-    t.slot = (p.first_frame[b] + fi) % p.C;
+    // frame list = the attended sink frames, then the recent frames
+    const int frame = fi < p.n_sink[b] ? fi : p.first_frame[b] + fi - p.n_sink[b];
+    t.slot = frame < p.sink ? frame : p.sink + (frame - p.sink) % p.C;
     t.tok0 = kTileN * tt;
   }
   return t;
@@ -851,9 +858,12 @@ using namespace unstep;
 typedef bool (*ScratchFn)(cudaStream_t st, size_t slots, size_t n_counters, Workspace* out);
 
 // Validation, work split, tensor maps and launch shared by the attention entry points.
+// The cache has `sink_frames` slots in front of the ring (0 for the plain rolling window);
+// stream b attends frames [0, min(sink_attend, lo)) and [lo, hi), lo = max(0, hi - window_frames).
 static int window_attn_run(const unstep_shape_t* shape, const int32_t* start_frame,
                            int32_t window_frames, const void* q_rot, const void* ring_k,
-                           const void* ring_v, void* out, void* cuda_stream, ScratchFn scratch) {
+                           const void* ring_v, void* out, void* cuda_stream, ScratchFn scratch,
+                           int32_t sink_frames = 0, int32_t sink_attend = 0) {
   int rc = check_shape(shape, true);
   if (rc != UNSTEP_OK) return rc;
   const void* ptrs[] = {start_frame, q_rot, ring_k, ring_v, out};
@@ -863,6 +873,8 @@ static int window_attn_run(const unstep_shape_t* shape, const int32_t* start_fra
     return UNSTEP_ERR_INVALID_ARG;
   if (window_frames < shape->chunk_frames || window_frames > shape->ring_frames)
     return UNSTEP_ERR_INVALID_ARG;
+  if (sink_frames < 0 || sink_frames > 4096 || sink_attend < 0 || sink_attend > sink_frames)
+    return UNSTEP_ERR_INVALID_ARG;
   for (int b = 0; b < shape->batch; ++b)
     if (start_frame[b] < 0 || start_frame[b] > INT32_MAX - shape->chunk_frames)
       return UNSTEP_ERR_INVALID_ARG;
@@ -871,13 +883,15 @@ static int window_attn_run(const unstep_shape_t* shape, const int32_t* start_fra
   const DeviceInfo& info = device_info();
   if (!info.ok) return UNSTEP_ERR_CUDA;
 
-  const uint64_t Hn = shape->heads, C = shape->ring_frames;
+  const uint64_t Hn = shape->heads;
+  const uint64_t C = static_cast<uint64_t>(shape->ring_frames) + sink_frames;  // cache slots per stream
   const uint64_t T = static_cast<uint64_t>(shape->grid_h) * shape->grid_w;
   const uint64_t L = T * shape->chunk_frames;
   const uint64_t row_bytes = Hn * kHeadDim * 2;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
 
   AttnParams p;
+  p.sink = sink_frames;
   p.Hn = shape->heads;
   p.L = static_cast<int32_t>(L);
   p.T = static_cast<int32_t>(T);
@@ -895,19 +909,31 @@ static int window_attn_run(const unstep_shape_t* shape, const int32_t* start_fra
     for (int i = 0; i < nb; ++i) {
       const int hi = start_frame[b0 + i] + shape->chunk_frames;
       const int lo = hi - window_frames > 0 ? hi - window_frames : 0;
+      const int n_sink = sink_attend < lo ? sink_attend : lo;   // sink frames not already in the recent part
       p.first_frame[i] = lo;
-      p.n_frames[i] = hi - lo;
+      p.n_sink[i] = n_sink;
+      for (int r = 0; r < 3; ++r) p.run_row0[i][r] = p.run_rows[i][r] = p.run_tile_end[i][r] = 0;
       if (p.flat) {
-        const int slot0 = lo % shape->ring_frames;
-        const int frames_a = (hi - lo) < shape->ring_frames - slot0 ? (hi - lo) : shape->ring_frames - slot0;
-        p.row0_a[i] = slot0 * p.T;
-        p.rows_a[i] = frames_a * p.T;
-        p.rows_b[i] = (hi - lo - frames_a) * p.T;
-        p.tiles_a[i] = (p.rows_a[i] + kTileN - 1) / kTileN;
-        p.tiles[i] = p.tiles_a[i] + (p.rows_b[i] + kTileN - 1) / kTileN;
+        // walk the attended frames in order and cut them into runs of consecutive cache slots
+        int n_runs = 0, prev_slot = -2;
+        for (int k = 0; k < n_sink + hi - lo; ++k) {
+          const int frame = k < n_sink ? k : lo + k - n_sink;
+          const int slot = frame < sink_frames ? frame : sink_frames + (frame - sink_frames) % shape->ring_frames;
+          if (slot != prev_slot + 1) {
+            if (n_runs == 3) return UNSTEP_ERR_INVALID_ARG;  // cannot happen: sink, ring end, ring start
+            p.run_row0[i][n_runs++] = slot * p.T;
+          }
+          p.run_rows[i][n_runs - 1] += p.T;
+          prev_slot = slot;
+        }
+        int tiles = 0;
+        for (int r = 0; r < 3; ++r) {
+          tiles += (p.run_rows[i][r] + kTileN - 1) / kTileN;
+          p.run_tile_end[i][r] = tiles;
+        }
+        p.tiles[i] = tiles;
       } else {
-        p.row0_a[i] = p.rows_a[i] = p.rows_b[i] = p.tiles_a[i] = 0;
-        p.tiles[i] = (hi - lo) * p.tiles_per_frame;
+        p.tiles[i] = (n_sink + hi - lo) * p.tiles_per_frame;
       }
     }
     // grid: one CTA per SM, fewer when the whole launch is small
@@ -966,6 +992,14 @@ extern "C" int unstep_window_attn(const unstep_shape_t* shape, const int32_t* st
                                   const void* ring_v, void* out, void* cuda_stream) {
   return window_attn_run(shape, start_frame, window_frames, q_rot, ring_k, ring_v, out, cuda_stream,
                          get_workspace);
+}
+
+extern "C" int unstep_window_attn_sink(const unstep_shape_t* shape, int32_t sink_frames,
+                                       const int32_t* start_frame, int32_t recent_frames,
+                                       int32_t sink_attend, const void* q_rot, const void* cache_k,
+                                       const void* cache_v, void* out, void* cuda_stream) {
+  return window_attn_run(shape, start_frame, recent_frames, q_rot, cache_k, cache_v, out, cuda_stream,
+                         get_workspace, sink_frames, sink_attend);
 }
 
 // --------------------------------------------------------------------------

@@ -45,11 +45,11 @@ __global__ void __launch_bounds__(256) rope_table_kernel(TableParams p, float* _
 // attention kernel right after, so they are left to the default cache policy.
 // --------------------------------------------------------------------------
 struct AppendParams {
-  int32_t L, T, C, vec_per_token;  // vec_per_token = Hn * 16
+  int32_t L, T, C, S, vec_per_token;  // C ring slots behind S sink slots; vec_per_token = Hn * 16
   int64_t vec_per_stream;          // L * Hn * 16
-  int64_t ring_vec_per_stream;     // C * T * Hn * 16
+  int64_t ring_vec_per_stream;     // (S + C) * T * Hn * 16
   int64_t table_stream_stride;     // elements
-  int32_t slot0[kMaxStreamsPerLaunch];  // start_frame[b] mod C
+  int32_t start[kMaxStreamsPerLaunch];  // start_frame[b]
 };
 
 __device__ __forceinline__ uint32_t rotate_pair(uint32_t w, float c, float s) {
@@ -82,8 +82,9 @@ rope_kv_append_kernel(AppendParams p, const uint4* q_in, const uint4* __restrict
   const int n = static_cast<int>(v / p.vec_per_token);
   const int rem = static_cast<int>(v - static_cast<int64_t>(n) * p.vec_per_token);
   const int f = n / p.T, t = n - f * p.T;
-  int slot = p.slot0[b] + f;
-  slot = slot % p.C;
+  // frames below S live in the sink prefix for good, later frames in the ring behind it
+  const int frame = p.start[b] + f;
+  const int slot = frame < p.S ? frame : p.S + (frame - p.S) % p.C;
 
   const int64_t in_idx = static_cast<int64_t>(b) * p.vec_per_stream + v;
   const uint4 xq = __ldcs(q_in + in_idx);
@@ -131,13 +132,14 @@ extern "C" int unstep_rope_table(const unstep_shape_t* shape, int32_t start_fram
   return cudaGetLastError() == cudaSuccess ? UNSTEP_OK : UNSTEP_ERR_CUDA;
 }
 
-extern "C" int unstep_rope_kv_append(const unstep_shape_t* shape, const int32_t* start_frame,
-                                     const void* q_in, const void* k_in, const void* v_in,
-                                     const float* cos, const float* sin,
-                                     int64_t table_stream_stride, void* q_out, void* ring_k,
-                                     void* ring_v, void* cuda_stream) {
+static int rope_kv_append_run(const unstep_shape_t* shape, int32_t sink_frames,
+                              const int32_t* start_frame, const void* q_in, const void* k_in,
+                              const void* v_in, const float* cos, const float* sin,
+                              int64_t table_stream_stride, void* q_out, void* ring_k, void* ring_v,
+                              void* cuda_stream) {
   int rc = check_shape(shape, true);
   if (rc != UNSTEP_OK) return rc;
+  if (sink_frames < 0 || sink_frames > 4096) return UNSTEP_ERR_INVALID_ARG;
   const void* ptrs[] = {start_frame, q_in, k_in, v_in, cos, sin, q_out, ring_k, ring_v};
   for (const void* ptr : ptrs)
     if (ptr == nullptr) return UNSTEP_ERR_INVALID_ARG;
@@ -146,7 +148,7 @@ extern "C" int unstep_rope_kv_append(const unstep_shape_t* shape, const int32_t*
     if (!aligned16(ptr)) return UNSTEP_ERR_INVALID_ARG;
   if (table_stream_stride < 0 || (table_stream_stride & 3)) return UNSTEP_ERR_INVALID_ARG;
   for (int b = 0; b < shape->batch; ++b)
-    if (start_frame[b] < 0) return UNSTEP_ERR_INVALID_ARG;
+    if (start_frame[b] < 0 || start_frame[b] > INT32_MAX - shape->chunk_frames) return UNSTEP_ERR_INVALID_ARG;
   rc = check_device();
   if (rc != UNSTEP_OK) return rc;
 
@@ -156,15 +158,16 @@ extern "C" int unstep_rope_kv_append(const unstep_shape_t* shape, const int32_t*
   p.L = static_cast<int32_t>(L);
   p.T = static_cast<int32_t>(T);
   p.C = shape->ring_frames;
+  p.S = sink_frames;
   p.vec_per_token = shape->heads * 16;
   p.vec_per_stream = L * p.vec_per_token;
-  p.ring_vec_per_stream = static_cast<int64_t>(shape->ring_frames) * T * p.vec_per_token;
+  p.ring_vec_per_stream = (static_cast<int64_t>(shape->ring_frames) + sink_frames) * T * p.vec_per_token;
   p.table_stream_stride = table_stream_stride;
   const unsigned blocks = static_cast<unsigned>((p.vec_per_stream + 255) / 256);
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   for (int b0 = 0; b0 < shape->batch; b0 += kMaxStreamsPerLaunch) {
     const int nb = shape->batch - b0 < kMaxStreamsPerLaunch ? shape->batch - b0 : kMaxStreamsPerLaunch;
-    for (int i = 0; i < nb; ++i) p.slot0[i] = start_frame[b0 + i] % shape->ring_frames;
+    for (int i = 0; i < nb; ++i) p.start[i] = start_frame[b0 + i];
     const int64_t in_off = static_cast<int64_t>(b0) * p.vec_per_stream;
     const int64_t ring_off = static_cast<int64_t>(b0) * p.ring_vec_per_stream;
     const int64_t tab_off = static_cast<int64_t>(b0) * table_stream_stride;
@@ -177,4 +180,22 @@ extern "C" int unstep_rope_kv_append(const unstep_shape_t* shape, const int32_t*
     if (cudaGetLastError() != cudaSuccess) return UNSTEP_ERR_CUDA;
   }
   return UNSTEP_OK;
+}
+
+extern "C" int unstep_rope_kv_append(const unstep_shape_t* shape, const int32_t* start_frame,
+                                     const void* q_in, const void* k_in, const void* v_in,
+                                     const float* cos, const float* sin,
+                                     int64_t table_stream_stride, void* q_out, void* ring_k,
+                                     void* ring_v, void* cuda_stream) {
+  return rope_kv_append_run(shape, 0, start_frame, q_in, k_in, v_in, cos, sin, table_stream_stride,
+                            q_out, ring_k, ring_v, cuda_stream);
+}
+
+extern "C" int unstep_rope_kv_append_sink(const unstep_shape_t* shape, int32_t sink_frames,
+                                          const int32_t* start_frame, const void* q_in,
+                                          const void* k_in, const void* v_in, const float* cos,
+                                          const float* sin, int64_t table_stream_stride, void* q_out,
+                                          void* cache_k, void* cache_v, void* cuda_stream) {
+  return rope_kv_append_run(shape, sink_frames, start_frame, q_in, k_in, v_in, cos, sin,
+                            table_stream_stride, q_out, cache_k, cache_v, cuda_stream);
 }

@@ -29,10 +29,11 @@ def abi_shape(sh: W.Shape) -> U.Shape:
 class DevicePath:
     """Device buffers of one layer and the calls on them."""
 
-    def __init__(self, sh: W.Shape, use_oracle_table: bool = True):
+    def __init__(self, sh: W.Shape, use_oracle_table: bool = True, sink_frames: int = 0):
         self.sh = sh
         self.abi = abi_shape(sh)
-        ring_shape = (sh.batch, sh.ring_frames, sh.tokens_per_frame, sh.heads, sh.head_dim)
+        self.sink = sink_frames
+        ring_shape = (sh.batch, sink_frames + sh.ring_frames, sh.tokens_per_frame, sh.heads, sh.head_dim)
         fill = torch.tensor(SENTINEL, dtype=torch.int16)
         self.ring_k = torch.full(ring_shape, int(fill), dtype=torch.int16, device="cuda").view(torch.bfloat16)
         self.ring_v = torch.full(ring_shape, int(fill), dtype=torch.int16, device="cuda").view(torch.bfloat16)
@@ -65,9 +66,19 @@ class DevicePath:
             stride = self.sh.chunk_tokens * 64
         q = to_dev(q_bits)
         q_out = q if in_place else torch.empty_like(q)
-        U.rope_kv_append(self.abi, starts, q, to_dev(k_bits), to_dev(v_bits), cos, sin, q_out,
-                         self.ring_k, self.ring_v, table_stream_stride=stride)
+        if self.sink:
+            U.rope_kv_append_sink(self.abi, self.sink, starts, q, to_dev(k_bits), to_dev(v_bits), cos, sin,
+                                  q_out, self.ring_k, self.ring_v, table_stream_stride=stride)
+        else:
+            U.rope_kv_append(self.abi, starts, q, to_dev(k_bits), to_dev(v_bits), cos, sin, q_out,
+                             self.ring_k, self.ring_v, table_stream_stride=stride)
         return q_out
+
+    def attend_sink(self, starts, recent_frames: int, sink_attend: int, q_rot: torch.Tensor) -> torch.Tensor:
+        out = torch.full_like(q_rot.view(torch.int16), SENTINEL).view(torch.bfloat16)
+        U.window_attn_sink(self.abi, self.sink, [int(s) for s in starts], recent_frames, sink_attend,
+                           q_rot, self.ring_k, self.ring_v, out)
+        return out
 
     def attend(self, starts, window_frames: int, q_rot: torch.Tensor) -> torch.Tensor:
         out = torch.full_like(q_rot.view(torch.int16), SENTINEL).view(torch.bfloat16)
