@@ -53,11 +53,17 @@ class Workload:
     window_frames: tuple         # window lengths (frames, chunk included) to attend with
     k_scale: float = 1.0
     note: str = ""
+    sink_frames: int = 0         # slots of the never-evicted prefix (0 = plain rolling window)
+    sink_attend: int = 0         # sink frames attended
 
     def keys_attended(self, window_frames: int):
         fc = self.shape.chunk_frames
-        return [min(window_frames, s + fc) * self.shape.tokens_per_frame
-                for s in self.measured_starts]
+        out = []
+        for s in self.measured_starts:
+            hi = s + fc
+            lo = max(0, hi - window_frames)
+            out.append((min(self.sink_attend, lo) + hi - lo) * self.shape.tokens_per_frame)
+        return out
 
     def attn_flops(self, window_frames: int) -> float:
         sh = self.shape
@@ -99,6 +105,16 @@ WORKLOADS = {
                      seed=4, history_starts=((0, 3, 6),), measured_starts=(9,),
                      window_frames=(12,)),
 }
+
+
+# the paper's operating point: 3 sink + 6 recent frames = 14040 keys, last chunk of a 21-frame clip
+WORKLOADS["cfg2_sink9"] = Workload("cfg2_sink9", replace(_S13, ring_frames=6), seed=5,
+                                   history_starts=(tuple(range(0, 18, 3)),), measured_starts=(18,),
+                                   window_frames=(6,), sink_frames=3, sink_attend=3)
+# the last chunk of a 30 s clip (123 latent frames) through the same 9-frame cache
+WORKLOADS["cfg2_sink9_long"] = Workload("cfg2_sink9_long", replace(_S13, ring_frames=6), seed=6,
+                                        history_starts=(tuple(range(0, 120, 3)),), measured_starts=(120,),
+                                        window_frames=(6,), sink_frames=3, sink_attend=3)
 
 
 def f32_to_bf16_bits(x: np.ndarray) -> np.ndarray:
