@@ -10,10 +10,12 @@
 // and O += P V accumulate in TMEM; P (bf16) is written back over S and fed to the
 // second MMA straight from TMEM.
 //
-// Keys are walked frame by frame: frame p of the window lives in ring slot p mod C and
-// every key tile lies inside one frame, so the 5-D tensor map (d, head, token, slot,
-// stream) zero-fills the ragged end of a frame and the ring is never copied.  The last
-// tile of a frame runs with a narrower MMA (N rounded up to 16).
+// The attended frames are at most three runs of consecutive cache slots (sink prefix, ring
+// up to its end, ring from its start).  Key tiles are cut from the runs through a flat
+// tensor map over cache rows; only the last tile of a run is ragged, and it is fetched
+// through a (token, slot) map whose zero fill ends it exactly at the end of its frame, so
+// the cache is never copied and slots outside the window may hold anything.  A ragged tile
+// runs with a narrower MMA (N and K rounded up to 16).
 #include <cuda.h>
 #include <cuda_bf16.h>
 
@@ -560,9 +562,10 @@ window_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
             tc_fence_after();
             issue_pv_half(dv, 0, k_steps, j > 0);
             issue_pv_half(dv, 1, k_steps, true);
-            tc_commit(bar_kv_empty + 8 * vst);
             TRACE(2 + a, sp_it, 4);
+            // the next S first (it is what the softmax warps wait for), the stage releases after it
             if (more) issue_qk(kst, valid);
+            tc_commit(bar_kv_empty + 8 * vst);
             TRACE(2 + a, sp_it, 5);
             ++sp_it;
           } else {
