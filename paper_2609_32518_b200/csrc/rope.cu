@@ -15,28 +15,56 @@ struct TableParams {
   double base;
 };
 
-__global__ void __launch_bounds__(256) rope_table_kernel(TableParams p, float* __restrict__ cos_out,
-                                                         float* __restrict__ sin_out) {
-  const int idx = blockIdx.x * blockDim.x + threadIdx.x;
-  if (idx >= p.L * kPairs) return;
-  const int n = idx >> 6, j = idx & 63;
-  const int T = p.grid_h * p.grid_w;
-  const int f = n / T, t = n - f * T;
-  const int r = t / p.grid_w, c = t - r * p.grid_w;
-  int i, d, pos;
-  if (j < p.pairs_t) {
-    i = j; d = p.band_t; pos = p.start_frame + f;
-  } else if (j < p.pairs_t + p.pairs_h) {
-    i = j - p.pairs_t; d = p.band_h; pos = r;
-  } else {
-    i = j - p.pairs_t - p.pairs_h; d = p.band_w; pos = c;
-  }
-  const double omega = pow(p.base, -(2.0 * static_cast<double>(i)) / static_cast<double>(d));
-  const double theta = static_cast<double>(pos) * omega;
+// cos and sin of position * omega in double, rounded once.
+__device__ __forceinline__ float2 table_entry(double omega, int pos) {
   double sn, cs;
-  sincos(theta, &sn, &cs);
-  cos_out[idx] = static_cast<float>(cs);
-  sin_out[idx] = static_cast<float>(sn);
+  sincos(static_cast<double>(pos) * omega, &sn, &cs);
+  return make_float2(static_cast<float>(cs), static_cast<float>(sn));
+}
+
+// One block per (frame, token row).  The table is separable: a token's 64 coefficients are
+// 22 that depend on its frame only, 21 on its row only and 21 on its column only.  The block
+// evaluates those (22 + 21 + 21 * grid_w double-precision values) once into shared memory and
+// then writes its grid_w * 64 entries of cos and sin with coalesced stores (64 columns per pass).  Evaluating every
+// entry on its own costs 64 double pow/sincos per token instead of about 22.
+__global__ void __launch_bounds__(1024) rope_table_kernel(TableParams p, float* __restrict__ cos_out,
+                                                         float* __restrict__ sin_out) {
+  constexpr int kColsPerPass = 64;
+  __shared__ float2 band[kPairs + kColsPerPass * kPairs];   // frame/row part, then [column][pair]
+  __shared__ double omega[kPairs];                          // base^(-2i/d_band) of the 64 pairs
+  const int r = blockIdx.x, f = blockIdx.y;
+  const int pairs_w = kPairs - p.pairs_t - p.pairs_h;
+  const int n_fixed = p.pairs_t + p.pairs_h;
+  if (threadIdx.x < kPairs) {
+    const int j = threadIdx.x;
+    const int i = j < p.pairs_t ? j : (j < n_fixed ? j - p.pairs_t : j - n_fixed);
+    const int d = j < p.pairs_t ? p.band_t : (j < n_fixed ? p.band_h : p.band_w);
+    omega[j] = pow(p.base, -(2.0 * static_cast<double>(i)) / static_cast<double>(d));
+  }
+  __syncthreads();
+  const int64_t row_base = (static_cast<int64_t>(f) * p.grid_h + r) * p.grid_w * kPairs;
+  for (int c0 = 0; c0 < p.grid_w; c0 += kColsPerPass) {
+    const int cols = min(kColsPerPass, p.grid_w - c0);
+    const int n_eval = n_fixed + cols * pairs_w;
+    for (int e = threadIdx.x; e < n_eval; e += blockDim.x) {
+      if (e < p.pairs_t) {
+        band[e] = table_entry(omega[e], p.start_frame + f);
+      } else if (e < n_fixed) {
+        band[e] = table_entry(omega[e], r);
+      } else {
+        const int c = (e - n_fixed) / pairs_w, i = (e - n_fixed) - c * pairs_w;
+        band[e] = table_entry(omega[n_fixed + i], c0 + c);
+      }
+    }
+    __syncthreads();
+    for (int idx = threadIdx.x; idx < cols * kPairs; idx += blockDim.x) {
+      const int c = idx >> 6, j = idx & 63;
+      const float2 v = j < n_fixed ? band[j] : band[n_fixed + c * pairs_w + (j - n_fixed)];
+      cos_out[row_base + c0 * kPairs + idx] = v.x;
+      sin_out[row_base + c0 * kPairs + idx] = v.y;
+    }
+    __syncthreads();
+  }
 }
 
 // --------------------------------------------------------------------------
@@ -125,9 +153,9 @@ extern "C" int unstep_rope_table(const unstep_shape_t* shape, int32_t start_fram
   p.band_h = shape->band_h;
   p.band_w = shape->band_w;
   p.base = shape->rope_base;
-  const int64_t total = static_cast<int64_t>(p.L) * kPairs;
-  const unsigned blocks = static_cast<unsigned>((total + 255) / 256);
-  rope_table_kernel<<<blocks, 256, 0, static_cast<cudaStream_t>(cuda_stream)>>>(p, cos_out, sin_out);
+  if (shape->chunk_frames > 65535) return UNSTEP_ERR_INVALID_ARG;
+  rope_table_kernel<<<dim3(shape->grid_h, shape->chunk_frames), 1024, 0,
+                      static_cast<cudaStream_t>(cuda_stream)>>>(p, cos_out, sin_out);
   g_launches.fetch_add(1);
   return cudaGetLastError() == cudaSuccess ? UNSTEP_OK : UNSTEP_ERR_CUDA;
 }
