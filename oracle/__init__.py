@@ -34,4 +34,6 @@ from .unstep_oracle import (  # noqa: F401
     rope_kv_append_sink,
     window_attn_sink,
     explicit_frames_attn,
+    rmsnorm_tokens,
+    rmsnorm_rope_kv_append,
 )

@@ -402,3 +402,36 @@ def explicit_frames_attn(history: ExplicitHistory, frames, q_rot_bits: np.ndarra
         v = bf16_bits_to_f32(v_bits[:, h]).astype(np.float64)
         out[:, hi_] = attention_rows(q, k, v)
     return out
+
+
+# ---------------------------------------------------------------------------
+# RMS normalisation of q and k in front of the rotation (appendix "Diffusion transformer
+# runtime": queries and keys are reshaped into heads "after linear projection and RMS
+# normalization").  The paper gives no formula; this is the textbook RMSNorm over the whole
+# token vector (all heads, Hn*128 wide) with a learned per-channel gain:
+#     y = x / sqrt(mean(x^2) + eps) * g
+# Readings: the mean of squares is accumulated in float64 (so that it does not depend on the
+# order of summation) and rounded to float32; sqrt, reciprocal and the two products are single
+# float32 operations; the result is rounded to bf16 (the tensor the rotation loads is bf16).
+# ---------------------------------------------------------------------------
+
+def rmsnorm_tokens(x_bits: np.ndarray, gain: np.ndarray, eps: float) -> np.ndarray:
+    """x_bits: bf16 bits [..., Hn, 128]; gain: float32 [Hn*128].  Returns bf16 bits."""
+    x = bf16_bits_to_f32(x_bits)
+    lead = x.shape[:-2]
+    width = x.shape[-2] * x.shape[-1]
+    flat = x.reshape(lead + (width,))
+    ms = (flat.astype(np.float64) ** 2).sum(axis=-1) / np.float64(width)
+    ms32 = ms.astype(np.float32)
+    r = (np.float32(1.0) / np.sqrt((ms32 + np.float32(eps)).astype(np.float32))).astype(np.float32)
+    y = ((flat * r[..., None]).astype(np.float32) * np.asarray(gain, dtype=np.float32)).astype(np.float32)
+    return f32_to_bf16_bits_rne(y).reshape(x_bits.shape)
+
+
+def rmsnorm_rope_kv_append(state, start_frames, q_bits, k_bits, v_bits, gain_q, gain_k, eps, cos, sin):
+    """RMSNorm of q and k, then the append (plain ring or sink cache, by the type of `state`)."""
+    qn = rmsnorm_tokens(q_bits, gain_q, eps)
+    kn = rmsnorm_tokens(k_bits, gain_k, eps)
+    if isinstance(state, SinkRingState):
+        return rope_kv_append_sink(state, start_frames, qn, kn, v_bits, cos, sin)
+    return rope_kv_append(state, start_frames, qn, kn, v_bits, cos, sin)
