@@ -150,6 +150,24 @@ int unstep_window_attn_sink(const unstep_shape_t* shape, int32_t sink_frames,
                             void* cuda_stream);
 
 /*
+ * RMS normalisation of q and k fused in front of the rotation (appendix "Diffusion transformer
+ * runtime": queries and keys are split into heads "after linear projection and RMS
+ * normalization"; the paper gives no formula, this is the textbook RMSNorm over the whole token
+ * vector of Hn*128 channels with a learned gain):
+ *     y = x / sqrt(mean(x^2) + eps) * gain,   rounded to bf16, then rotated and appended exactly
+ * as unstep_rope_kv_append_sink does (v is copied, not normalised).  The mean of squares is
+ * accumulated in double and rounded to float32; sqrt, reciprocal and the two products are single
+ * float32 operations.  Saves one read and one write of q and k compared with a separate norm.
+ *   gain_q, gain_k : float32 [Hn*128], read.     eps : >= 0.
+ *   sink_frames    : 0 for the plain ring.  All other arguments as in unstep_rope_kv_append_sink.
+ */
+int unstep_rmsnorm_rope_kv_append(const unstep_shape_t* shape, int32_t sink_frames,
+                                  const int32_t* start_frame, const void* q_in, const void* k_in,
+                                  const void* v_in, const float* gain_q, const float* gain_k, float eps,
+                                  const float* cos, const float* sin, int64_t table_stream_stride,
+                                  void* q_out, void* cache_k, void* cache_v, void* cuda_stream);
+
+/*
  * unstep_window_attn for callers that must not allocate.  (The paper has no counterpart:
  * this is a deployment variant of the call above, same arguments, same result.)
  *

@@ -14,6 +14,7 @@ from .binding import (  # noqa: F401
     window_attn_noalloc,
     rope_kv_append_sink,
     window_attn_sink,
+    rmsnorm_rope_kv_append,
     poll_status,
     launch_count,
     strerror,

@@ -3,13 +3,13 @@
 from __future__ import annotations
 
 import ctypes
-from ctypes import c_char_p, c_double, c_int, c_int32, c_int64, c_void_p, POINTER
+from ctypes import c_char_p, c_double, c_float, c_int, c_int32, c_int64, c_void_p, POINTER
 
 from . import build as _build
 
 EXPORTS = ("unstep_rope_table", "unstep_rope_kv_append", "unstep_window_attn",
            "unstep_window_attn_noalloc", "unstep_rope_kv_append_sink", "unstep_window_attn_sink",
-           "unstep_strerror", "unstep_poll_status", "unstep_launch_count")
+           "unstep_rmsnorm_rope_kv_append", "unstep_strerror", "unstep_poll_status", "unstep_launch_count")
 
 
 class UnstepError(RuntimeError):
@@ -67,6 +67,11 @@ def lib() -> ctypes.CDLL:
         L.unstep_window_attn_sink.restype = c_int
         L.unstep_window_attn_sink.argtypes = [POINTER(Shape), c_int32, POINTER(c_int32), c_int32, c_int32,
                                               c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]
+        L.unstep_rmsnorm_rope_kv_append.restype = c_int
+        L.unstep_rmsnorm_rope_kv_append.argtypes = [POINTER(Shape), c_int32, POINTER(c_int32), c_void_p,
+                                                    c_void_p, c_void_p, c_void_p, c_void_p, c_float,
+                                                    c_void_p, c_void_p, c_int64, c_void_p, c_void_p,
+                                                    c_void_p, c_void_p]
         L.unstep_strerror.restype = c_char_p
         L.unstep_strerror.argtypes = [c_int]
         L.unstep_poll_status.restype = c_int
@@ -184,6 +189,26 @@ def rope_kv_append_sink(shape: Shape, sink_frames: int, start_frame, q_in, k_in,
         _dev_ptr(cos, torch.float32, ntab, "cos"), _dev_ptr(sin, torch.float32, ntab, "sin"),
         int(table_stream_stride), _dev_ptr(q_out, bf, n, "q_out"), _dev_ptr(cache_k, bf, nr, "cache_k"),
         _dev_ptr(cache_v, bf, nr, "cache_v"), _stream_ptr(stream)), "unstep_rope_kv_append_sink")
+
+
+def rmsnorm_rope_kv_append(shape: Shape, sink_frames: int, start_frame, q_in, k_in, v_in, gain_q, gain_k,
+                           eps: float, cos, sin, q_out, cache_k, cache_v, table_stream_stride: int = 0,
+                           stream=None):
+    """unstep_rmsnorm_rope_kv_append: RMSNorm of q and k, rotation and cache write in one kernel."""
+    import torch
+    bf = torch.bfloat16
+    n = shape.batch * shape.chunk_tokens * shape.heads * shape.head_dim
+    nr = (shape.batch * (shape.ring_frames + int(sink_frames)) * shape.tokens_per_frame * shape.heads
+          * shape.head_dim)
+    ntab = shape.chunk_tokens * 64 + (shape.batch - 1) * int(table_stream_stride)
+    ng = shape.heads * shape.head_dim
+    _check(lib().unstep_rmsnorm_rope_kv_append(
+        ctypes.byref(shape), int(sink_frames), _starts(shape, start_frame),
+        _dev_ptr(q_in, bf, n, "q_in"), _dev_ptr(k_in, bf, n, "k_in"), _dev_ptr(v_in, bf, n, "v_in"),
+        _dev_ptr(gain_q, torch.float32, ng, "gain_q"), _dev_ptr(gain_k, torch.float32, ng, "gain_k"),
+        c_float(eps), _dev_ptr(cos, torch.float32, ntab, "cos"), _dev_ptr(sin, torch.float32, ntab, "sin"),
+        int(table_stream_stride), _dev_ptr(q_out, bf, n, "q_out"), _dev_ptr(cache_k, bf, nr, "cache_k"),
+        _dev_ptr(cache_v, bf, nr, "cache_v"), _stream_ptr(stream)), "unstep_rmsnorm_rope_kv_append")
 
 
 def window_attn_sink(shape: Shape, sink_frames: int, start_frame, recent_frames: int, sink_attend: int,

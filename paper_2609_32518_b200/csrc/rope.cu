@@ -130,6 +130,110 @@ rope_kv_append_kernel(AppendParams p, const uint4* q_in, const uint4* __restrict
   ring_v[ring_idx] = xv;
 }
 
+// --------------------------------------------------------------------------
+// RMSNorm of q and k fused in front of the rotation: one warp per token.  The norm runs over
+// the whole token vector (all heads).  Pass 1 loads the token's q and k vectors and sums their
+// squares in double (exact for bf16 data, so the order of summation does not matter); pass 2
+// normalises (float32: sqrt, reciprocal and two products, each rounded once), rounds to bf16 as
+// the unfused pipeline would, rotates and stores.  Up to 8 vectors per lane stay in registers
+// between the passes; wider tokens are read again (from L1/L2).
+// --------------------------------------------------------------------------
+constexpr int kNormCached = 8;
+
+__device__ __forceinline__ double warp_sum(double x) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xFFFFFFFFu, x, o);
+  return x;
+}
+__device__ __forceinline__ double squares(uint4 x) {
+  double s = 0.0;
+  const uint32_t w[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const float lo = __uint_as_float(w[i] << 16), hi = __uint_as_float(w[i] & 0xFFFF0000u);
+    s += static_cast<double>(lo * lo) + static_cast<double>(hi * hi);   // bf16 squares are exact in float
+  }
+  return s;
+}
+// y = bf16(fl32(fl32(x * r) * g)) for the 8 elements of a vector
+__device__ __forceinline__ uint4 normalise_vec(uint4 x, float r, float4 g0, float4 g1) {
+  const uint32_t w[4] = {x.x, x.y, x.z, x.w};
+  const float g[8] = {g0.x, g0.y, g0.z, g0.w, g1.x, g1.y, g1.z, g1.w};
+  uint32_t y[4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const float lo = __fmul_rn(__fmul_rn(__uint_as_float(w[i] << 16), r), g[2 * i]);
+    const float hi = __fmul_rn(__fmul_rn(__uint_as_float(w[i] & 0xFFFF0000u), r), g[2 * i + 1]);
+    const __nv_bfloat162 b = __floats2bfloat162_rn(lo, hi);
+    y[i] = *reinterpret_cast<const uint32_t*>(&b);
+  }
+  return make_uint4(y[0], y[1], y[2], y[3]);
+}
+
+template <bool kCached>
+__global__ void __launch_bounds__(256)
+rmsnorm_rope_kv_append_kernel(AppendParams p, float eps, const uint4* q_in, const uint4* __restrict__ k_in,
+                              const uint4* __restrict__ v_in, const float4* __restrict__ gain_q,
+                              const float4* __restrict__ gain_k, const float4* __restrict__ cos_t,
+                              const float4* __restrict__ sin_t, uint4* q_out, uint4* __restrict__ ring_k,
+                              uint4* __restrict__ ring_v) {
+  const int b = blockIdx.y;
+  const int lane = threadIdx.x & 31;
+  const int n = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);   // token of this warp
+  if (n >= p.L) return;
+  const int f = n / p.T, t = n - f * p.T;
+  const int frame = p.start[b] + f;
+  const int slot = frame < p.S ? frame : p.S + (frame - p.S) % p.C;
+  const int64_t in_base = static_cast<int64_t>(b) * p.vec_per_stream + static_cast<int64_t>(n) * p.vec_per_token;
+  const int64_t ring_base = static_cast<int64_t>(b) * p.ring_vec_per_stream +
+                            (static_cast<int64_t>(slot) * p.T + t) * p.vec_per_token;
+  const int64_t tab_base = (static_cast<int64_t>(b) * p.table_stream_stride >> 2) +
+                           static_cast<int64_t>(n) * (kPairs / 4);
+
+  uint4 cq[kCached ? kNormCached : 1], ck[kCached ? kNormCached : 1];
+  double sq = 0.0, sk = 0.0;
+  if (kCached) {
+#pragma unroll
+    for (int u = 0; u < kNormCached; ++u) {
+      const int vi = lane + 32 * u;
+      if (vi < p.vec_per_token) {
+        cq[u] = __ldcs(q_in + in_base + vi);
+        ck[u] = __ldcs(k_in + in_base + vi);
+        sq += squares(cq[u]);
+        sk += squares(ck[u]);
+      }
+    }
+  } else {
+    for (int vi = lane; vi < p.vec_per_token; vi += 32) {
+      sq += squares(q_in[in_base + vi]);   // plain load: q_out may be the same buffer
+      sk += squares(__ldg(k_in + in_base + vi));
+    }
+  }
+  const double width = static_cast<double>(p.vec_per_token) * 8.0;
+  const float ms_q = static_cast<float>(warp_sum(sq) / width), ms_k = static_cast<float>(warp_sum(sk) / width);
+  const float rq = __frcp_rn(__fsqrt_rn(__fadd_rn(ms_q, eps)));
+  const float rk = __frcp_rn(__fsqrt_rn(__fadd_rn(ms_k, eps)));
+
+  auto finish = [&](int vi, uint4 xq, uint4 xk) {
+    const float4 c = __ldg(cos_t + tab_base + (vi & 15));
+    const float4 s = __ldg(sin_t + tab_base + (vi & 15));
+    const uint4 nq = normalise_vec(xq, rq, __ldg(gain_q + 2 * vi), __ldg(gain_q + 2 * vi + 1));
+    const uint4 nk = normalise_vec(xk, rk, __ldg(gain_k + 2 * vi), __ldg(gain_k + 2 * vi + 1));
+    q_out[in_base + vi] = rotate_vec(nq, c, s);
+    ring_k[ring_base + vi] = rotate_vec(nk, c, s);
+    ring_v[ring_base + vi] = __ldcs(v_in + in_base + vi);
+  };
+  if (kCached) {
+#pragma unroll
+    for (int u = 0; u < kNormCached; ++u) {
+      const int vi = lane + 32 * u;
+      if (vi < p.vec_per_token) finish(vi, cq[u], ck[u]);
+    }
+  } else {
+    for (int vi = lane; vi < p.vec_per_token; vi += 32) finish(vi, q_in[in_base + vi], k_in[in_base + vi]);
+  }
+}
+
 }  // namespace unstep
 
 using namespace unstep;
@@ -226,4 +330,65 @@ extern "C" int unstep_rope_kv_append_sink(const unstep_shape_t* shape, int32_t s
                                           void* cache_k, void* cache_v, void* cuda_stream) {
   return rope_kv_append_run(shape, sink_frames, start_frame, q_in, k_in, v_in, cos, sin,
                             table_stream_stride, q_out, cache_k, cache_v, cuda_stream);
+}
+
+extern "C" int unstep_rmsnorm_rope_kv_append(const unstep_shape_t* shape, int32_t sink_frames,
+                                             const int32_t* start_frame, const void* q_in,
+                                             const void* k_in, const void* v_in, const float* gain_q,
+                                             const float* gain_k, float eps, const float* cos,
+                                             const float* sin, int64_t table_stream_stride, void* q_out,
+                                             void* cache_k, void* cache_v, void* cuda_stream) {
+  int rc = check_shape(shape, true);
+  if (rc != UNSTEP_OK) return rc;
+  if (sink_frames < 0 || sink_frames > 4096 || !(eps >= 0.f)) return UNSTEP_ERR_INVALID_ARG;
+  const void* ptrs[] = {start_frame, q_in, k_in, v_in, gain_q, gain_k, cos, sin, q_out, cache_k, cache_v};
+  for (const void* ptr : ptrs)
+    if (ptr == nullptr) return UNSTEP_ERR_INVALID_ARG;
+  const void* dev_ptrs[] = {q_in, k_in, v_in, gain_q, gain_k, cos, sin, q_out, cache_k, cache_v};
+  for (const void* ptr : dev_ptrs)
+    if (!aligned16(ptr)) return UNSTEP_ERR_INVALID_ARG;
+  if (table_stream_stride < 0 || (table_stream_stride & 3)) return UNSTEP_ERR_INVALID_ARG;
+  for (int b = 0; b < shape->batch; ++b)
+    if (start_frame[b] < 0 || start_frame[b] > INT32_MAX - shape->chunk_frames) return UNSTEP_ERR_INVALID_ARG;
+  rc = check_device();
+  if (rc != UNSTEP_OK) return rc;
+
+  const int64_t T = static_cast<int64_t>(shape->grid_h) * shape->grid_w;
+  const int64_t L = T * shape->chunk_frames;
+  AppendParams p;
+  p.L = static_cast<int32_t>(L);
+  p.T = static_cast<int32_t>(T);
+  p.C = shape->ring_frames;
+  p.S = sink_frames;
+  p.vec_per_token = shape->heads * 16;
+  p.vec_per_stream = L * p.vec_per_token;
+  p.ring_vec_per_stream = (static_cast<int64_t>(shape->ring_frames) + sink_frames) * T * p.vec_per_token;
+  p.table_stream_stride = table_stream_stride;
+  const unsigned blocks = static_cast<unsigned>((L + 7) / 8);   // 8 warps = 8 tokens per block
+  const bool cached = p.vec_per_token <= 32 * kNormCached;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  for (int b0 = 0; b0 < shape->batch; b0 += kMaxStreamsPerLaunch) {
+    const int nb = shape->batch - b0 < kMaxStreamsPerLaunch ? shape->batch - b0 : kMaxStreamsPerLaunch;
+    for (int i = 0; i < nb; ++i) p.start[i] = start_frame[b0 + i];
+    const int64_t in_off = static_cast<int64_t>(b0) * p.vec_per_stream;
+    const int64_t ring_off = static_cast<int64_t>(b0) * p.ring_vec_per_stream;
+    const int64_t tab_off = static_cast<int64_t>(b0) * table_stream_stride;
+    const uint4* q = static_cast<const uint4*>(q_in) + in_off;
+    const uint4* k = static_cast<const uint4*>(k_in) + in_off;
+    const uint4* v = static_cast<const uint4*>(v_in) + in_off;
+    const float4* gq = reinterpret_cast<const float4*>(gain_q);
+    const float4* gk = reinterpret_cast<const float4*>(gain_k);
+    const float4* ct = reinterpret_cast<const float4*>(cos + tab_off);
+    const float4* sn = reinterpret_cast<const float4*>(sin + tab_off);
+    uint4* qo = static_cast<uint4*>(q_out) + in_off;
+    uint4* rk = static_cast<uint4*>(cache_k) + ring_off;
+    uint4* rv = static_cast<uint4*>(cache_v) + ring_off;
+    if (cached)
+      rmsnorm_rope_kv_append_kernel<true><<<dim3(blocks, nb), 256, 0, st>>>(p, eps, q, k, v, gq, gk, ct, sn, qo, rk, rv);
+    else
+      rmsnorm_rope_kv_append_kernel<false><<<dim3(blocks, nb), 256, 0, st>>>(p, eps, q, k, v, gq, gk, ct, sn, qo, rk, rv);
+    g_launches.fetch_add(1);
+    if (cudaGetLastError() != cudaSuccess) return UNSTEP_ERR_CUDA;
+  }
+  return UNSTEP_OK;
 }
