@@ -204,11 +204,17 @@ def run_ours(args):
         for b, sb in enumerate(s if tab_stride else s[:1]):
             U.rope_table(abi, sb, cos[b], sin[b])
 
+    gain_q = 1.0 + 0.1 * torch.randn(sh.heads * sh.head_dim, device=dev, generator=gen)
+    gain_k = 1.0 + 0.1 * torch.randn(sh.heads * sh.head_dim, device=dev, generator=gen)
+
     def append(q, k, v):
         c_, s_ = (cos, sin) if tab_stride else (cos[0], sin[0])
         if tab_stride == 0:
             c_, s_ = c_.contiguous(), s_.contiguous()
-        if sink:
+        if args.rmsnorm:
+            U.rmsnorm_rope_kv_append(abi, sink, s, q, k, v, gain_q, gain_k, 1e-6, c_, s_, q_rot, ring_k, ring_v,
+                                     table_stream_stride=tab_stride)
+        elif sink:
             U.rope_kv_append_sink(abi, sink, s, q, k, v, c_, s_, q_rot, ring_k, ring_v, table_stream_stride=tab_stride)
         else:
             U.rope_kv_append(abi, s, q, k, v, c_, s_, q_rot, ring_k, ring_v, table_stream_stride=tab_stride)
@@ -332,7 +338,7 @@ def run_ours(args):
                      "frac_of_sustained": attn_tflops / peaks["bf16_tflops_sustained"],
                      "frac_of_nominal_2250": attn_tflops / 2250.0,
                      "traffic": ATTN_DRAM_TRAFFIC_BYTES},
-        "append_roofline": {"kernel": "rope_kv_append_kernel", "bound": "hbm",
+        "append_roofline": {"kernel": "rmsnorm_rope_kv_append_kernel" if args.rmsnorm else "rope_kv_append_kernel", "bound": "hbm",
                             "achieved": append_bytes / (t_append * 1e-3) / 1e9, "peak": peaks["hbm_gbs"],
                             "unit": "GB/s", "frac": append_bytes / (t_append * 1e-3) / 1e9 / peaks["hbm_gbs"],
                             "peak_source": f"{peaks['source']} copy", "bytes": append_bytes},
@@ -365,6 +371,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--workload", default=WORKLOAD, choices=sorted(W.WORKLOADS),
                     help="configuration to time (default: the 1.3B-class shape the metric is quoted on)")
+    ap.add_argument("--rmsnorm", action="store_true",
+                    help="use the append with the q/k RMS norm fused in (not the default path)")
     ap.add_argument("--window", type=int, default=0, help="window length in frames (default: the workload's)")
     args = ap.parse_args()
     if args.impl == "reference":

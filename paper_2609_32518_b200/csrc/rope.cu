@@ -135,25 +135,33 @@ rope_kv_append_kernel(AppendParams p, const uint4* q_in, const uint4* __restrict
 // the whole token vector (all heads).  Pass 1 loads the token's q and k vectors and sums their
 // squares in double (exact for bf16 data, so the order of summation does not matter); pass 2
 // normalises (float32: sqrt, reciprocal and two products, each rounded once), rounds to bf16 as
-// the unfused pipeline would, rotates and stores.  Up to 8 vectors per lane stay in registers
-// between the passes; wider tokens are read again (from L1/L2).
+// the unfused pipeline would, rotates and stores.  Pass 2 reads q and k again, from L1/L2:
+// keeping them in registers between the passes cost more in occupancy than the second read.
 // --------------------------------------------------------------------------
-constexpr int kNormCached = 8;
 
 __device__ __forceinline__ double warp_sum(double x) {
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xFFFFFFFFu, x, o);
   return x;
 }
+// Exact widening of a non-negative float to double with integer operations (the conversion
+// instruction is a slow-rate one): rebias the exponent, move the mantissa.  Zero and float
+// denormals take the ordinary conversion.
+__device__ __forceinline__ double widen_nonneg(float v) {
+  const uint32_t u = __float_as_uint(v);
+  if ((u & 0x7F800000u) == 0u) return static_cast<double>(v);
+  return __hiloint2double(static_cast<int>((u >> 3) + 0x38000000u), static_cast<int>(u << 29));
+}
 __device__ __forceinline__ double squares(uint4 x) {
-  double s = 0.0;
+  double s0 = 0.0, s1 = 0.0;
   const uint32_t w[4] = {x.x, x.y, x.z, x.w};
 #pragma unroll
   for (int i = 0; i < 4; ++i) {
     const float lo = __uint_as_float(w[i] << 16), hi = __uint_as_float(w[i] & 0xFFFF0000u);
-    s += static_cast<double>(lo * lo) + static_cast<double>(hi * hi);   // bf16 squares are exact in float
+    s0 += widen_nonneg(lo * lo);   // a bf16 square has 16 significant bits: exact in float
+    s1 += widen_nonneg(hi * hi);
   }
-  return s;
+  return s0 + s1;
 }
 // y = bf16(fl32(fl32(x * r) * g)) for the 8 elements of a vector
 __device__ __forceinline__ uint4 normalise_vec(uint4 x, float r, float4 g0, float4 g1) {
@@ -170,7 +178,6 @@ __device__ __forceinline__ uint4 normalise_vec(uint4 x, float r, float4 g0, floa
   return make_uint4(y[0], y[1], y[2], y[3]);
 }
 
-template <bool kCached>
 __global__ void __launch_bounds__(256)
 rmsnorm_rope_kv_append_kernel(AppendParams p, float eps, const uint4* q_in, const uint4* __restrict__ k_in,
                               const uint4* __restrict__ v_in, const float4* __restrict__ gain_q,
@@ -190,23 +197,26 @@ rmsnorm_rope_kv_append_kernel(AppendParams p, float eps, const uint4* q_in, cons
   const int64_t tab_base = (static_cast<int64_t>(b) * p.table_stream_stride >> 2) +
                            static_cast<int64_t>(n) * (kPairs / 4);
 
-  uint4 cq[kCached ? kNormCached : 1], ck[kCached ? kNormCached : 1];
   double sq = 0.0, sk = 0.0;
-  if (kCached) {
+  {
+    // four vectors of q and of k per lane in flight at a time
+    for (int v0 = lane; v0 < p.vec_per_token; v0 += 32 * 4) {
+      uint4 xq[4], xk[4];
 #pragma unroll
-    for (int u = 0; u < kNormCached; ++u) {
-      const int vi = lane + 32 * u;
-      if (vi < p.vec_per_token) {
-        cq[u] = __ldcs(q_in + in_base + vi);
-        ck[u] = __ldcs(k_in + in_base + vi);
-        sq += squares(cq[u]);
-        sk += squares(ck[u]);
+      for (int u = 0; u < 4; ++u) {
+        const int vi = v0 + 32 * u;
+        if (vi < p.vec_per_token) {
+          xq[u] = q_in[in_base + vi];   // plain load: q_out may be the same buffer
+          xk[u] = __ldg(k_in + in_base + vi);
+        }
       }
-    }
-  } else {
-    for (int vi = lane; vi < p.vec_per_token; vi += 32) {
-      sq += squares(q_in[in_base + vi]);   // plain load: q_out may be the same buffer
-      sk += squares(__ldg(k_in + in_base + vi));
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        if (v0 + 32 * u < p.vec_per_token) {
+          sq += squares(xq[u]);
+          sk += squares(xk[u]);
+        }
+      }
     }
   }
   const double width = static_cast<double>(p.vec_per_token) * 8.0;
@@ -223,14 +233,21 @@ rmsnorm_rope_kv_append_kernel(AppendParams p, float eps, const uint4* q_in, cons
     ring_k[ring_base + vi] = rotate_vec(nk, c, s);
     ring_v[ring_base + vi] = __ldcs(v_in + in_base + vi);
   };
-  if (kCached) {
+  {
+    for (int v0 = lane; v0 < p.vec_per_token; v0 += 32 * 2) {
+      uint4 xq[2], xk[2];
 #pragma unroll
-    for (int u = 0; u < kNormCached; ++u) {
-      const int vi = lane + 32 * u;
-      if (vi < p.vec_per_token) finish(vi, cq[u], ck[u]);
+      for (int u = 0; u < 2; ++u) {
+        const int vi = v0 + 32 * u;
+        if (vi < p.vec_per_token) {
+          xq[u] = q_in[in_base + vi];
+          xk[u] = k_in[in_base + vi];
+        }
+      }
+#pragma unroll
+      for (int u = 0; u < 2; ++u)
+        if (v0 + 32 * u < p.vec_per_token) finish(v0 + 32 * u, xq[u], xk[u]);
     }
-  } else {
-    for (int vi = lane; vi < p.vec_per_token; vi += 32) finish(vi, q_in[in_base + vi], k_in[in_base + vi]);
   }
 }
 
@@ -365,7 +382,6 @@ extern "C" int unstep_rmsnorm_rope_kv_append(const unstep_shape_t* shape, int32_
   p.ring_vec_per_stream = (static_cast<int64_t>(shape->ring_frames) + sink_frames) * T * p.vec_per_token;
   p.table_stream_stride = table_stream_stride;
   const unsigned blocks = static_cast<unsigned>((L + 7) / 8);   // 8 warps = 8 tokens per block
-  const bool cached = p.vec_per_token <= 32 * kNormCached;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   for (int b0 = 0; b0 < shape->batch; b0 += kMaxStreamsPerLaunch) {
     const int nb = shape->batch - b0 < kMaxStreamsPerLaunch ? shape->batch - b0 : kMaxStreamsPerLaunch;
@@ -383,10 +399,7 @@ extern "C" int unstep_rmsnorm_rope_kv_append(const unstep_shape_t* shape, int32_
     uint4* qo = static_cast<uint4*>(q_out) + in_off;
     uint4* rk = static_cast<uint4*>(cache_k) + ring_off;
     uint4* rv = static_cast<uint4*>(cache_v) + ring_off;
-    if (cached)
-      rmsnorm_rope_kv_append_kernel<true><<<dim3(blocks, nb), 256, 0, st>>>(p, eps, q, k, v, gq, gk, ct, sn, qo, rk, rv);
-    else
-      rmsnorm_rope_kv_append_kernel<false><<<dim3(blocks, nb), 256, 0, st>>>(p, eps, q, k, v, gq, gk, ct, sn, qo, rk, rv);
+    rmsnorm_rope_kv_append_kernel<<<dim3(blocks, nb), 256, 0, st>>>(p, eps, q, k, v, gq, gk, ct, sn, qo, rk, rv);
     g_launches.fetch_add(1);
     if (cudaGetLastError() != cudaSuccess) return UNSTEP_ERR_CUDA;
   }
