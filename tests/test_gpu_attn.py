@@ -116,3 +116,26 @@ def test_cfg4_clean_cache_pattern():
 
 def test_cfg5_sampled_rows():
     run(W.WORKLOADS["cfg5"], rows_fn=lambda L: W.sample_rows(L, per_tile=2), heads=[0, 13, 39])
+
+
+def test_more_streams_than_one_launch_carries():
+    # 35 streams (the per-launch parameter block holds 32), one short frame per chunk, own positions
+    sh = W.Shape(batch=35, heads=1, chunk_frames=1, grid_h=4, grid_w=10, ring_frames=4)
+    starts = tuple(3 + (b % 5) for b in range(35))
+    wl = W.Workload("many", sh, seed=24, history_starts=((),) * 35, measured_starts=starts,
+                    window_frames=(4, 2, 1))
+    dev, ora = DevicePath(sh), OraclePath(sh)
+    for back in (3, 2, 1):                       # frames start-3 .. start-1 of every stream
+        prev = [s - back for s in starts]
+        q, k, v = W.batch_qkv(wl, prev)
+        dev.append(prev, q, k, v)
+        ora.append(prev, q, k, v)
+    run(wl, dev=dev, ora=ora)
+
+
+def test_queries_shorter_than_a_tile_and_single_head():
+    # L = 2*3*5 = 30 queries, T = 15 keys per frame: one ragged query tile, per-frame key tiles
+    sh = W.Shape(batch=2, heads=1, chunk_frames=2, grid_h=3, grid_w=5, ring_frames=6)
+    wl = W.Workload("short", sh, seed=25, history_starts=((0, 2, 4), (0,)), measured_starts=(6, 2),
+                    window_frames=(6, 3, 2), k_scale=4.0)
+    run(wl)

@@ -111,3 +111,23 @@ def test_sink_argument_checks():
     assert L.unstep_window_attn_sink(ctypes.byref(sh), -1, one, 6, 0, f, f, f, f, None) == -1
     assert L.unstep_window_attn_sink(ctypes.byref(sh), 3, one, 7, 3, f, f, f, f, None) == -1   # recent > ring
     assert L.unstep_rope_kv_append_sink(ctypes.byref(sh), -2, one, f, f, f, f, f, 0, f, f, f, None) == -1
+
+
+def test_short_frames_sink_cache_per_frame_tiles():
+    # T = 6*7 = 42 keys per frame (< one tile): the per-frame addressing with a sink prefix
+    sh = W.Shape(batch=2, heads=2, chunk_frames=3, grid_h=6, grid_w=7, ring_frames=6)
+    wl = W.Workload("short_sink", sh, seed=53, history_starts=((), ()), measured_starts=(0, 0),
+                    window_frames=(6,), k_scale=4.0)
+    dev = DevicePath(sh, sink_frames=2)
+    ora = O.SinkRingState(2, 2, 6, sh.tokens_per_frame, sh.heads)
+    for c in range(9):
+        starts = [3 * c, 3 * c]
+        q, k, v = W.batch_qkv(wl, starts)
+        cos, sin = tables(sh, 3 * c)
+        q_dev = dev.append(starts, q, k, v)
+        q_ref = O.rope_kv_append_sink(ora, starts, q, k, v, cos, sin)
+        assert np.array_equal(to_bits(dev.ring_k), ora.cache_k)
+        for sink_attend in (2, 1):
+            out = to_bits(dev.attend_sink(starts, 6, sink_attend, q_dev))
+            check(out, O.window_attn_sink(ora, starts, 6, sink_attend, q_ref, 3), f"chunk {c} sink {sink_attend}")
+    assert U.poll_status() == 0
