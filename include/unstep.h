@@ -116,6 +116,10 @@ int unstep_rope_kv_append(const unstep_shape_t* shape, const int32_t* start_fram
  *                   been appended and not yet overwritten (true when chunks arrive in
  *                   order and window_frames <= C).
  *   out           : bf16 [B, L, Hn, 128], written.
+ * Scratch: work items that are split across thread blocks exchange partial results through a
+ * buffer the library keeps per (device, stream).  The first call on a stream creates it with
+ * cudaMalloc (about 40 MB): make that call outside any stream capture.  Calls on one stream
+ * share the buffer safely; calls on different streams use different buffers.
  */
 int unstep_window_attn(const unstep_shape_t* shape, const int32_t* start_frame,
                        int32_t window_frames, const void* q_rot, const void* ring_k,
