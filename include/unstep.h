@@ -213,6 +213,15 @@ const char* unstep_strerror(int code);
  */
 int unstep_poll_status(void);
 
+/*
+ * Self-test of the bounded device-side waits: launches one small kernel that waits, with the same
+ * code the attention kernel uses, on a barrier that nothing signals, gives up after `limit_cycles`
+ * SM clock cycles (1 .. 4e9), records UNSTEP_ERR_TIMEOUT in the status word and returns normally.
+ * Nothing traps or hangs; the context stays usable.  Afterwards unstep_poll_status() returns
+ * UNSTEP_ERR_TIMEOUT once.
+ */
+int unstep_selftest_wait_limit(int64_t limit_cycles, void* cuda_stream);
+
 /* Number of kernels the library has launched in this process (all devices). */
 int64_t unstep_launch_count(void);
 

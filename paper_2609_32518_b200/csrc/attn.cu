@@ -215,6 +215,7 @@ __device__ __forceinline__ void named_barrier_128(int id) {
 
 struct Waiter {
   volatile int* abort_flag;
+  long long limit;   // clock cycles after which a wait gives up
   // Bounded wait: the hardware parks the thread between polls; the clock and the CTA's abort
   // flag are only looked at every 32 polls so that a waiting warp leaves the issue slots alone.
   __device__ __forceinline__ bool wait(uint32_t bar, uint32_t parity) const {
@@ -224,7 +225,7 @@ struct Waiter {
       if (mbar_try_wait_hint(bar, parity, 2000u)) return true;
       if ((spin & 31u) == 0u) {
         if (*abort_flag) return false;
-        if (clock64() - t0 > kWaitCycles) {
+        if (clock64() - t0 > limit) {
           *abort_flag = 1;
           atomicExch(&g_status, UNSTEP_ERR_TIMEOUT);
           return false;
@@ -430,7 +431,7 @@ window_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
-  const Waiter w{abort_flag};
+  const Waiter w{abort_flag, kWaitCycles};
 
   if (warp >= 8) {
     reg_dealloc_96();
@@ -742,6 +743,22 @@ window_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
   }
   __syncthreads();
   if (warp == 8) tmem_dealloc(tmem_base, kTmemCols);
+}
+
+// A wait on a barrier that nothing ever arrives at, with a short limit: exercises the give-up
+// path of Waiter (status word, flag, orderly return) without any other work.
+__global__ void wait_limit_probe_kernel(long long limit_cycles) {
+  __shared__ __align__(8) uint64_t bar;
+  __shared__ int abort_flag;
+  if (threadIdx.x == 0) {
+    mbar_init(smem_u32(&bar), 1);
+    abort_flag = 0;
+    mbar_fence_init();
+  }
+  __syncthreads();
+  const Waiter w{&abort_flag, limit_cycles};
+  w.wait(smem_u32(&bar), 0);
+  __syncthreads();
 }
 
 // --------------------------------------------------------------------------
@@ -1071,6 +1088,15 @@ extern "C" int unstep_window_attn_noalloc(const unstep_shape_t* shape, const int
   if (info.sm_count > kStaticMaxCtas) return UNSTEP_ERR_TOO_LARGE;
   return window_attn_run(shape, start_frame, window_frames, q_rot, ring_k, ring_v, out, cuda_stream,
                          static_scratch);
+}
+
+extern "C" int unstep_selftest_wait_limit(int64_t limit_cycles, void* cuda_stream) {
+  if (limit_cycles < 1 || limit_cycles > 4000000000LL) return UNSTEP_ERR_INVALID_ARG;
+  const int rc = check_device();
+  if (rc != UNSTEP_OK) return rc;
+  wait_limit_probe_kernel<<<1, 64, 0, static_cast<cudaStream_t>(cuda_stream)>>>(limit_cycles);
+  g_launches.fetch_add(1);
+  return cudaGetLastError() == cudaSuccess ? UNSTEP_OK : UNSTEP_ERR_CUDA;
 }
 
 extern "C" int unstep_poll_status(void) {
