@@ -325,7 +325,8 @@ def run_ours(args):
     ms_step = total_ms / K
     t_table = float(np.mean([e[0].elapsed_time(e[1]) for e in evs]))
     t_append = float(np.mean([e[1].elapsed_time(e[2]) for e in evs]))
-    t_attn = float(np.mean([e[2].elapsed_time(e[3]) for e in evs]))
+    attn_times = np.array([e[2].elapsed_time(e[3]) for e in evs])
+    t_attn = float(attn_times.mean())
     status = U.poll_status()
 
     # ---- end to end: pinned host inputs in, result back to the host, every step ---------
@@ -362,6 +363,7 @@ def run_ours(args):
         "us_per_layer_chunk": ms_step * 1e3,
         "kernels_us": {"rope_table": t_table * 1e3, "rope_kv_append": t_append * 1e3,
                        "window_attn": t_attn * 1e3},
+        "window_attn_us_median_min": [float(np.median(attn_times)) * 1e3, float(attn_times.min()) * 1e3],
         "roofline": {"kernel": "window_attn_kernel", "bound": "tensor", "achieved": attn_tflops,
                      "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
                      "frac": attn_tflops / peaks["bf16_tflops"],

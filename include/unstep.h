@@ -222,6 +222,12 @@ int unstep_poll_status(void);
  */
 int unstep_selftest_wait_limit(int64_t limit_cycles, void* cuda_stream);
 
+/*
+ * Optional: waits for the devices to go idle and frees the scratch buffers unstep_window_attn
+ * created (all devices, all streams).  The library stays usable; the next call makes new ones.
+ */
+void unstep_shutdown(void);
+
 /* Number of kernels the library has launched in this process (all devices). */
 int64_t unstep_launch_count(void);
 

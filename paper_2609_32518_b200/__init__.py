@@ -16,6 +16,7 @@ from .binding import (  # noqa: F401
     window_attn_sink,
     rmsnorm_rope_kv_append,
     poll_status,
+    shutdown,
     selftest_wait_limit,
     launch_count,
     strerror,

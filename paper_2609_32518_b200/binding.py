@@ -9,7 +9,7 @@ from . import build as _build
 
 EXPORTS = ("unstep_rope_table", "unstep_rope_kv_append", "unstep_window_attn",
            "unstep_window_attn_noalloc", "unstep_rope_kv_append_sink", "unstep_window_attn_sink",
-           "unstep_rmsnorm_rope_kv_append", "unstep_selftest_wait_limit", "unstep_strerror", "unstep_poll_status", "unstep_launch_count")
+           "unstep_rmsnorm_rope_kv_append", "unstep_selftest_wait_limit", "unstep_shutdown", "unstep_strerror", "unstep_poll_status", "unstep_launch_count")
 
 
 class UnstepError(RuntimeError):
@@ -74,6 +74,8 @@ def lib() -> ctypes.CDLL:
                                                     c_void_p, c_void_p]
         L.unstep_selftest_wait_limit.restype = c_int
         L.unstep_selftest_wait_limit.argtypes = [c_int64, c_void_p]
+        L.unstep_shutdown.restype = None
+        L.unstep_shutdown.argtypes = []
         L.unstep_strerror.restype = c_char_p
         L.unstep_strerror.argtypes = [c_int]
         L.unstep_poll_status.restype = c_int
@@ -232,6 +234,11 @@ def selftest_wait_limit(limit_cycles: int, stream=None):
     """unstep_selftest_wait_limit: make a bounded device-side wait run out (diagnostic)."""
     _check(lib().unstep_selftest_wait_limit(int(limit_cycles), _stream_ptr(stream)),
            "unstep_selftest_wait_limit")
+
+
+def shutdown():
+    """unstep_shutdown: free the scratch buffers the attention calls created."""
+    lib().unstep_shutdown()
 
 
 def poll_status() -> int:

@@ -1099,6 +1099,22 @@ extern "C" int unstep_selftest_wait_limit(int64_t limit_cycles, void* cuda_strea
   return cudaGetLastError() == cudaSuccess ? UNSTEP_OK : UNSTEP_ERR_CUDA;
 }
 
+extern "C" void unstep_shutdown(void) {
+  // frees the per-stream scratch buffers of every device; the next attention call makes new ones
+  cudaDeviceSynchronize();
+  int cur = 0;
+  if (cudaGetDevice(&cur) != cudaSuccess) return;
+  std::lock_guard<std::mutex> lock(g_ws_mutex);
+  for (auto& kv : g_workspaces) {
+    if (cudaSetDevice(kv.first.first) != cudaSuccess) continue;
+    cudaDeviceSynchronize();
+    if (kv.second.part != nullptr) cudaFree(kv.second.part);
+    if (kv.second.counters != nullptr) cudaFree(kv.second.counters);
+  }
+  g_workspaces.clear();
+  cudaSetDevice(cur);
+}
+
 extern "C" int unstep_poll_status(void) {
   if (cudaDeviceSynchronize() != cudaSuccess) return UNSTEP_ERR_CUDA;
   int st = 0, zero = 0;

@@ -29,3 +29,12 @@ def test_limit_argument_is_checked():
         U.selftest_wait_limit(0)
     with pytest.raises(U.UnstepError):
         U.selftest_wait_limit(5_000_000_000)
+
+
+def test_shutdown_frees_scratch_and_the_library_keeps_working():
+    run(W.WORKLOADS["cfg1_wrapped"])
+    before = torch.cuda.mem_get_info()[0]
+    U.shutdown()
+    after = torch.cuda.mem_get_info()[0]
+    assert after >= before                      # the scratch (tens of MB) went back to the driver
+    run(W.WORKLOADS["cfg1_wrapped"])            # and is made again on demand
