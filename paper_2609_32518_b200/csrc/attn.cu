@@ -908,6 +908,7 @@ static int window_attn_run(const unstep_shape_t* shape, const int32_t* start_fra
   const uint64_t T = static_cast<uint64_t>(shape->grid_h) * shape->grid_w;
   const uint64_t L = T * shape->chunk_frames;
   const uint64_t row_bytes = Hn * kHeadDim * 2;
+  if (C * T >= (uint64_t(1) << 30)) return UNSTEP_ERR_INVALID_ARG;  // cache rows are 32-bit coordinates
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
 
   AttnParams p;
