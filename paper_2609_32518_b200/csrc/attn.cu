@@ -35,6 +35,16 @@ __device__ int g_status = 0;
 // Optional timeline of CTA 0 (debug builds only): clock64 stamps per role, tile and event.
 #ifdef UNSTEP_TRACE
 __device__ long long g_trace[4][64][8];
+__device__ unsigned long long g_cta_trace[160][16];
+__device__ __forceinline__ unsigned long long gtime() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+  return t;
+}
+#define CTRACE(ev)                                                                       \
+  do {                                                                                   \
+    if (threadIdx.x == 0 && (ev) < 16) g_cta_trace[blockIdx.x][ev] = gtime();            \
+  } while (0)
 #define TRACE(role, tile, ev)                                                          \
   do {                                                                                 \
     if (blockIdx.x == 0 && (tile) < 64 && (threadIdx.x == 0 || threadIdx.x == 256 || threadIdx.x == 288)) g_trace[role][tile][ev] = clock64(); \
@@ -42,6 +52,9 @@ __device__ long long g_trace[4][64][8];
 #else
 #define TRACE(role, tile, ev) \
   do {                        \
+  } while (0)
+#define CTRACE(ev) \
+  do {             \
   } while (0)
 #endif
 
@@ -406,6 +419,7 @@ window_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
   const int tid = threadIdx.x;
   const int warp = tid >> 5;
   const int lane = tid & 31;
+  CTRACE(0);
 
   if (tid == 0) {
     for (int i = 0; i < 2; ++i) {
@@ -591,6 +605,8 @@ window_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
     Seg s;
     uint32_t it[2] = {0, 0}, seg_it[2] = {0, 0}, x_it = 0;
     bool ok = true;
+    int seg_no = 0;
+    CTRACE(1);
     while (ok && sched.next(s)) {
       float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};
       for (int j = s.t0; j < s.t1 && ok; ++j) {
@@ -602,6 +618,7 @@ window_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
           TRACE(a, it[a], 0);
           w.wait(bar_s_full + 8 * a, it[a] & 1);  // on failure the flag is up: handled after the barrier
           tc_fence_after();
+          if (it[0] == 0) CTRACE(2);
           TRACE(a, it[a], 1);
           volatile float* xc = xchg + (x_it & 1) * 256;
           const uint32_t t_S = t_lane + a * 128, t_O = t_lane + 256 + a * 128;
@@ -618,11 +635,12 @@ window_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         }
       }
       if (!ok) break;
-      // epilogue of both query tiles
-      for (int a = 0; a < s.nq && ok; ++a) {
+      CTRACE(8 + seg_no);
+      // ---- epilogue of the segment: both query tiles' accumulators are final ----
+      float l_all[2] = {0.f, 0.f};
+      for (int a = 0; a < s.nq; ++a) {
         w.wait(bar_o_final + 8 * a, seg_it[a] & 1);
         ++seg_it[a];
-        tc_fence_after();
         // row sum = the two partners' partial sums
         volatile float* xc = xchg + (x_it & 1) * 256;
         ++x_it;
@@ -632,103 +650,139 @@ window_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
           ok = false;
           break;
         }
-        const float l_all = l_run[a] + xc[(1 - half) * 128 + row];
-        const uint32_t t_O = t_lane + 256 + a * 128 + 64 * half;
+        l_all[a] = l_run[a] + xc[(1 - half) * 128 + row];
+      }
+      if (!ok) break;
+      tc_fence_after();
+      const bool whole = (s.t0 == 0 && s.t1 == s.tiles);
+      // this thread's 64 output columns of row n of query tile a
+      auto out_ptr = [&](int a) -> uint4* {
         const int n = (2 * s.qp + a) * kTileM + row;
-        uint4* dst = reinterpret_cast<uint4*>(
+        return reinterpret_cast<uint4*>(
             out + ((static_cast<int64_t>(s.b) * p.L + n) * p.Hn + s.h) * kHeadDim + 64 * half);
-        const bool whole = (s.t0 == 0 && s.t1 == s.tiles);
-        if (whole) {
-          // O / l -> bf16 -> out[b][n][h][64*half ...]
-          const float inv_l = 1.f / l_all;
+      };
+      auto store_row = [&](uint4* dst, const float* v, float inv_l) {   // 32 columns
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          uint4 vv;
+          vv.x = pack_bf16x2(v[8 * i + 0] * inv_l, v[8 * i + 1] * inv_l);
+          vv.y = pack_bf16x2(v[8 * i + 2] * inv_l, v[8 * i + 3] * inv_l);
+          vv.z = pack_bf16x2(v[8 * i + 4] * inv_l, v[8 * i + 5] * inv_l);
+          vv.w = pack_bf16x2(v[8 * i + 6] * inv_l, v[8 * i + 7] * inv_l);
+          dst[i] = vv;
+        }
+      };
+      if (whole) {
+        // O / l -> bf16 -> out[b][n][h][64*half ...]
+        for (int a = 0; a < s.nq; ++a) {
+          const uint32_t t_O = t_lane + 256 + a * 128 + 64 * half;
+          const bool in_range = (2 * s.qp + a) * kTileM + row < p.L;
+          const float inv_l = 1.f / l_all[a];
+          uint4* dst = out_ptr(a);
 #pragma unroll
           for (int q = 0; q < 2; ++q) {
-            uint32_t o[32];
-            tmem_ld32(t_O + q * 32, o);
+            float o[32];
+            tmem_ld32(t_O + q * 32, reinterpret_cast<uint32_t*>(o));
             tc_wait_ld();
-            if (n < p.L) {
+            if (in_range) store_row(dst + 4 * q, o, inv_l);
+          }
+        }
+      } else {
+        // Part of a split item.  The parts of an item are merged by whichever of them is done
+        // last, in part order (a fixed order, so the result does not depend on which one that
+        // is); the merging part takes its own accumulators straight from TMEM.  A part that
+        // finds all others already published merges at once without publishing itself;
+        // otherwise it publishes (O, m, l) of both tiles, counts itself in, and merges if
+        // that made the count complete.
+        const int c_lo = Sched::cta_of(p, s.item_step0);
+        const int c_hi = Sched::cta_of(p, s.item_step0 + s.tiles - 1);
+        const int others = c_hi - c_lo;
+        int* counter = p.counters + 2 * s.item;
+        if (tid == 0) {
+          int seen;
+          asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(seen) : "l"(counter) : "memory");
+          *merge_flag = (seen == others) ? 1 : 0;
+        }
+        softmax_barrier();
+        bool last = (*merge_flag != 0);
+        if (!last) {
+          float* mine = p.part + static_cast<int64_t>(2 * blockIdx.x + (s.first_in_cta ? 0 : 1)) * kPartFloats;
+          for (int a = 0; a < s.nq; ++a) {
+            const uint32_t t_O = t_lane + 256 + a * 128 + 64 * half;
+            float* dstp = mine + a * kPartTileFloats;
 #pragma unroll
-              for (int i = 0; i < 4; ++i) {
-                uint4 vv;
-                vv.x = pack_bf16x2(__uint_as_float(o[8 * i + 0]) * inv_l, __uint_as_float(o[8 * i + 1]) * inv_l);
-                vv.y = pack_bf16x2(__uint_as_float(o[8 * i + 2]) * inv_l, __uint_as_float(o[8 * i + 3]) * inv_l);
-                vv.z = pack_bf16x2(__uint_as_float(o[8 * i + 4]) * inv_l, __uint_as_float(o[8 * i + 5]) * inv_l);
-                vv.w = pack_bf16x2(__uint_as_float(o[8 * i + 6]) * inv_l, __uint_as_float(o[8 * i + 7]) * inv_l);
-                dst[q * 4 + i] = vv;
-              }
+            for (int q = 0; q < 2; ++q) {
+              uint32_t o[32];
+              tmem_ld32(t_O + q * 32, o);
+              tc_wait_ld();
+#pragma unroll
+              for (int i = 0; i < 32; ++i) dstp[(64 * half + q * 32 + i) * 128 + row] = __uint_as_float(o[i]);
+            }
+            if (half == 0) {
+              dstp[128 * 128 + row] = m_run[a];
+              dstp[128 * 128 + 128 + row] = l_all[a];
             }
           }
-        } else {
-          // part of a split item: publish (O, m, l), count the arrival; the last part to arrive
-          // merges all of them in part order (a fixed order, so the result does not depend on
-          // which CTA happens to be last)
-          float* mine = p.part + (static_cast<int64_t>(2 * blockIdx.x + (s.first_in_cta ? 0 : 1)) * kPartFloats +
-                                  a * kPartTileFloats);
-#pragma unroll
-          for (int q = 0; q < 2; ++q) {
-            uint32_t o[32];
-            tmem_ld32(t_O + q * 32, o);
-            tc_wait_ld();
-#pragma unroll
-            for (int i = 0; i < 32; ++i) mine[(64 * half + q * 32 + i) * 128 + row] = __uint_as_float(o[i]);
-          }
-          if (half == 0) {
-            mine[128 * 128 + row] = m_run[a];
-            mine[128 * 128 + 128 + row] = l_all;
-          }
           __threadfence();
+          softmax_barrier();   // all of this part is published; everyone has read the flag
+          if (tid == 0) *merge_flag = (atomicAdd(counter, 1) == others) ? 1 : 0;
           softmax_barrier();
-          const int c_lo = Sched::cta_of(p, s.item_step0);
-          const int c_hi = Sched::cta_of(p, s.item_step0 + s.tiles - 1);
-          if (tid == 0) *merge_flag = atomicAdd(p.counters + 2 * s.item + a, 1);
-          softmax_barrier();
-          const bool last = (*merge_flag == c_hi - c_lo);
-          softmax_barrier();  // everyone has read the flag before it can be written again
-          if (last) {
-            if (tid == 0) p.counters[2 * s.item + a] = 0;  // ready for the next launch
-            __threadfence();
+          last = (*merge_flag != 0);
+        }
+        if (last) {
+          __threadfence();
+          if (tid == 0) *counter = 0;   // ready for the next launch
+          const int me = static_cast<int>(blockIdx.x);
+          for (int a = 0; a < s.nq; ++a) {
             auto part_of = [&](int c) -> const float* {
               const int64_t clo = Sched::cta_lo(p, c);
               const bool first = clo >= s.item_step0;   // the part starts the range of CTA c
               return p.part + (static_cast<int64_t>(2 * c + (first ? 0 : 1)) * kPartFloats + a * kPartTileFloats);
             };
-            float m_all = -INFINITY;
-            for (int c = c_lo; c <= c_hi; ++c) m_all = fmaxf(m_all, __ldcg(part_of(c) + 128 * 128 + row));
+            const uint32_t t_O = t_lane + 256 + a * 128 + 64 * half;
+            float m_all = m_run[a];
+            for (int c = c_lo; c <= c_hi; ++c)
+              if (c != me) m_all = fmaxf(m_all, __ldcg(part_of(c) + 128 * 128 + row));
             float l_sum = 0.f;
             for (int c = c_lo; c <= c_hi; ++c) {
               const float* pc = part_of(c);
-              l_sum += __ldcg(pc + 128 * 128 + 128 + row) *
-                       ex2((__ldcg(pc + 128 * 128 + row) - m_all) * p.scale_log2e);
+              const float m_c = c == me ? m_run[a] : __ldcg(pc + 128 * 128 + row);
+              const float l_c = c == me ? l_all[a] : __ldcg(pc + 128 * 128 + 128 + row);
+              l_sum += l_c * ex2((m_c - m_all) * p.scale_log2e);
             }
             const float inv_l = 1.f / l_sum;
-#pragma unroll 1
-            for (int q = 0; q < 2; ++q) {
-              float acc[32];
+            float acc[64];
 #pragma unroll
-              for (int i = 0; i < 32; ++i) acc[i] = 0.f;
-              for (int c = c_lo; c <= c_hi; ++c) {
+            for (int i = 0; i < 64; ++i) acc[i] = 0.f;
+            for (int c = c_lo; c <= c_hi; ++c) {
+              float v[64];
+              float m_c;
+              if (c == me) {
+                tmem_ld32(t_O, reinterpret_cast<uint32_t*>(v));
+                tmem_ld32(t_O + 32, reinterpret_cast<uint32_t*>(v) + 32);
+                tc_wait_ld();
+                m_c = m_run[a];
+              } else {
                 const float* pc = part_of(c);
-                const float sc = ex2((__ldcg(pc + 128 * 128 + row) - m_all) * p.scale_log2e);
 #pragma unroll
-                for (int i = 0; i < 32; ++i)
-                  acc[i] = fmaf(__ldcg(pc + (64 * half + q * 32 + i) * 128 + row), sc, acc[i]);
+                for (int i = 0; i < 64; ++i) v[i] = __ldcg(pc + (64 * half + i) * 128 + row);
+                m_c = __ldcg(pc + 128 * 128 + row);
               }
-              if (n < p.L) {
+              const float sc = ex2((m_c - m_all) * p.scale_log2e);
 #pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                  uint4 vv;
-                  vv.x = pack_bf16x2(acc[8 * i + 0] * inv_l, acc[8 * i + 1] * inv_l);
-                  vv.y = pack_bf16x2(acc[8 * i + 2] * inv_l, acc[8 * i + 3] * inv_l);
-                  vv.z = pack_bf16x2(acc[8 * i + 4] * inv_l, acc[8 * i + 5] * inv_l);
-                  vv.w = pack_bf16x2(acc[8 * i + 6] * inv_l, acc[8 * i + 7] * inv_l);
-                  dst[q * 4 + i] = vv;
-                }
-              }
+              for (int i = 0; i < 64; ++i) acc[i] = fmaf(v[i], sc, acc[i]);
+            }
+            if ((2 * s.qp + a) * kTileM + row < p.L) {
+              uint4* dst = out_ptr(a);
+              store_row(dst, acc, inv_l);
+              store_row(dst + 4, acc + 32, inv_l);
             }
           }
         }
-        tc_fence_before();
       }
+      tc_fence_before();
+      CTRACE(3 + seg_no);
+      ++seg_no;
     }
   }
 
@@ -743,6 +797,7 @@ window_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
   }
   __syncthreads();
   if (warp == 8) tmem_dealloc(tmem_base, kTmemCols);
+  CTRACE(7);
 }
 
 // A wait on a barrier that nothing ever arrives at, with a short limit: exercises the give-up
@@ -1001,6 +1056,11 @@ static int window_attn_run(const unstep_shape_t* shape, const int32_t* start_fra
 }
 
 #ifdef UNSTEP_TRACE
+extern "C" int unstep_debug_read_cta_trace(unsigned long long* host_out) {
+  if (cudaDeviceSynchronize() != cudaSuccess) return UNSTEP_ERR_CUDA;
+  return cudaMemcpyFromSymbol(host_out, g_cta_trace, sizeof(unsigned long long) * 160 * 16) == cudaSuccess
+             ? UNSTEP_OK : UNSTEP_ERR_CUDA;
+}
 extern "C" int unstep_debug_read_trace(long long* host_out) {
   if (cudaDeviceSynchronize() != cudaSuccess) return UNSTEP_ERR_CUDA;
   return cudaMemcpyFromSymbol(host_out, g_trace, sizeof(long long) * 4 * 64 * 8) == cudaSuccess
