@@ -34,7 +34,7 @@ __device__ int g_status = 0;
 
 // Optional timeline of CTA 0 (debug builds only): clock64 stamps per role, tile and event.
 #ifdef UNSTEP_TRACE
-__device__ long long g_trace[4][64][8];
+__device__ long long g_trace[12][64][8];
 __device__ unsigned long long g_cta_trace[160][16];
 __device__ __forceinline__ unsigned long long gtime() {
   unsigned long long t;
@@ -47,7 +47,11 @@ __device__ __forceinline__ unsigned long long gtime() {
   } while (0)
 #define TRACE(role, tile, ev)                                                          \
   do {                                                                                 \
-    if (blockIdx.x == 0 && (tile) < 64 && (threadIdx.x == 0 || threadIdx.x == 256 || threadIdx.x == 288)) g_trace[role][tile][ev] = clock64(); \
+    if (blockIdx.x == 0 && (tile) < 64 && (threadIdx.x & 31) == 0) {                   \
+      const int w_ = threadIdx.x >> 5;                                                 \
+      const int slot_ = (role) < 2 ? (w_ & 3) * 2 + (role) : 8 + (role) - 2;            \
+      g_trace[slot_][tile][ev] = clock64();                                            \
+    }                                                                                  \
   } while (0)
 #else
 #define TRACE(role, tile, ev) \
@@ -229,6 +233,27 @@ __device__ __forceinline__ void named_barrier_128(int id) {
 struct Waiter {
   volatile int* abort_flag;
   long long limit;   // clock cycles after which a wait gives up
+  // Bounded wait that polls without parking the thread: for the single-lane roles on the
+  // critical path of a tile, where the wake-up of a parked thread would add to every hand-over.
+  __device__ __forceinline__ bool spin(uint32_t bar, uint32_t parity) const {
+#ifdef UNSTEP_NO_SPIN
+    return wait(bar, parity);
+#else
+    if (mbar_test_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    for (uint32_t n = 1;; ++n) {
+      if (mbar_test_wait(bar, parity)) return true;
+      if ((n & 1023u) == 0u) {
+        if (*abort_flag) return false;
+        if (clock64() - t0 > limit) {
+          *abort_flag = 1;
+          atomicExch(&g_status, UNSTEP_ERR_TIMEOUT);
+          return false;
+        }
+      }
+    }
+#endif
+  }
   // Bounded wait: the hardware parks the thread between polls; the clock and the CTA's abort
   // flag are only looked at every 32 polls so that a waiting warp leaves the issue slots alone.
   __device__ __forceinline__ bool wait(uint32_t bar, uint32_t parity) const {
@@ -248,6 +273,9 @@ struct Waiter {
   }
 };
 
+// The CTA owns 384 x 168 registers; 128 x 96 + 256 x 200 stays inside that (an increase that
+// the pool cannot satisfy would wait forever).
+static_assert(128 * 96 + 256 * 200 <= 384 * 168, "register redistribution exceeds the CTA's allocation");
 __device__ __forceinline__ void reg_dealloc_96() { asm volatile("setmaxnreg.dec.sync.aligned.u32 96;"); }
 __device__ __forceinline__ void reg_alloc_200() { asm volatile("setmaxnreg.inc.sync.aligned.u32 200;"); }
 
@@ -388,6 +416,154 @@ __device__ __forceinline__ bool softmax_tile(uint32_t t_S, uint32_t t_O, float c
   return true;
 }
 
+#ifndef UNSTEP_ROW_SOFTMAX
+#define UNSTEP_ROW_SOFTMAX 1
+#endif
+#ifndef UNSTEP_TURN_AT
+#define UNSTEP_TURN_AT 4
+#endif
+
+// --------------------------------------------------------------------------------------
+// Softmax of one 128 x 128 score tile with one thread per query row (a warpgroup per query
+// tile).  The two warpgroups run independently and drift half a period apart, so that one
+// is in its MUFU-bound exponentials while the other loads, reduces and stores, and the tensor
+// core works on one tile while the other is in its softmax.  No data crosses threads.
+// P is handed over in two halves of 64 keys, so P V can start on the first half.
+// --------------------------------------------------------------------------------------
+__device__ __forceinline__ void group_barrier(int a) {
+  if (a == 0) asm volatile("bar.sync 1, 128;" ::: "memory");
+  else asm volatile("bar.sync 2, 128;" ::: "memory");
+}
+
+// Exponentials of 32 score columns (registers s) into 16 bf16 pairs (p) and the packed sums.
+__device__ __forceinline__ void exp_block32(const uint32_t* s, uint32_t* p, uint64_t c2, uint64_t nm2,
+                                            uint64_t* acc) {
+#pragma unroll
+  for (int i = 0; i < 16; ++i) {
+    const uint64_t x2 = fma_f32x2(pack_f32x2(__uint_as_float(s[2 * i]), __uint_as_float(s[2 * i + 1])), c2, nm2);
+    float p0, p1;
+    if ((i & 7) < UNSTEP_EMU_OF8) {
+      // part of the exponentials runs on the FMA pipe: the MUFU pipe alone would bound the tile
+      exp2_poly_pair(x2, p0, p1);
+    } else {
+      float x0, x1;
+      unpack_f32x2(x2, x0, x1);
+      p0 = ex2(x0);
+      p1 = ex2(x1);
+    }
+    acc[i & 3] = add_f32x2(acc[i & 3], pack_f32x2(p0, p1));
+    p[i] = pack_bf16x2(p0, p1);
+  }
+}
+__device__ __forceinline__ float max_block32(const uint32_t* s) {
+  float m = fmaxf(__uint_as_float(s[0]), __uint_as_float(s[1]));
+#pragma unroll
+  for (int i = 2; i < 32; i += 2) m = max3(m, __uint_as_float(s[i]), __uint_as_float(s[i + 1]));
+  return m;
+}
+template <bool kMasked>
+__device__ __forceinline__ void mask_block32(uint32_t* s, int col0, int nvalid) {
+  if (kMasked) {
+#pragma unroll
+    for (int i = 0; i < 32; ++i)
+      if (col0 + i >= nvalid) s[i] = 0xFF800000u;  // -inf
+  }
+}
+
+// The scores are read from TMEM twice to keep the register count down: a first pass for the
+// row maximum (keys 64..127, then 0..63, the latter kept), then the exponentials of keys 0..63
+// from registers while keys 64..127 are fetched again in two blocks of 32.  P (bf16 pairs)
+// overwrites score columns 0..63, which are in registers by then.
+template <bool kMasked>
+__device__ __forceinline__ bool softmax_row_tile(uint32_t t_S, uint32_t t_O, float c, int nvalid,
+                                                 bool first, float& m_run, float& l_run,
+                                                 uint32_t bar_p_half, const Waiter& w, uint32_t turn_wait,
+                                                 uint32_t turn_parity, uint32_t turn_signal,
+                                                 int trace_role, int trace_tile) {
+  uint32_t lo[64];
+  float mx;
+  {
+    uint32_t hi[64];
+    tmem_ld32(t_S + 64, hi);
+    tmem_ld32(t_S + 96, hi + 32);
+    tmem_ld32(t_S, lo);
+    tmem_ld32(t_S + 32, lo + 32);
+    tc_wait_ld();
+    TRACE(trace_role, trace_tile, 2);
+    mask_block32<kMasked>(hi, 64, nvalid);
+    mask_block32<kMasked>(hi + 32, 96, nvalid);
+    mask_block32<kMasked>(lo, 0, nvalid);
+    mask_block32<kMasked>(lo + 32, 32, nvalid);
+    mx = fmaxf(fmaxf(max_block32(hi), max_block32(hi + 32)), fmaxf(max_block32(lo), max_block32(lo + 32)));
+  }
+  TRACE(trace_role, trace_tile, 3);
+  float alpha = 1.f;
+  bool grow = false;
+  if (first) {
+    m_run = mx;
+  } else if ((mx - m_run) * c > kRescaleThreshold) {
+    alpha = ex2((m_run - mx) * c);
+    m_run = mx;
+    l_run *= alpha;
+    grow = true;
+  }
+  if (__any_sync(0xFFFFFFFFu, grow)) {
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      uint32_t o[32];
+      tmem_ld32(t_O + q * 32, o);
+      tc_wait_ld();
+#pragma unroll
+      for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
+      tmem_st32(t_O + q * 32, o);
+    }
+  }
+  // The two warpgroups take turns on the exponentials: the MUFU pipe is shared, and alternating
+  // keeps the two query tiles half a period apart, so that the tensor pipe has one tile's MMAs
+  // to run while the other tile is in its softmax.
+  if (turn_wait != 0u && !w.wait(turn_wait, turn_parity)) return false;
+  TRACE(trace_role, trace_tile, 6);
+  // p = 2^(s*c - m*c): packed FMA on pairs, MUFU or polynomial, packed partial sums
+  const uint64_t c2 = pack_f32x2(c, c);
+  const float neg_ms = -m_run * c;
+  const uint64_t nm2 = pack_f32x2(neg_ms, neg_ms);
+  uint64_t acc[4] = {0ull, 0ull, 0ull, 0ull};
+  uint32_t h0[32], h1[32];
+  tmem_ld32(t_S + 64, h0);             // keys 64..95 again, in flight during the first half
+  {
+    uint32_t preg[32];
+    exp_block32(lo, preg, c2, nm2, acc);
+    exp_block32(lo + 32, preg + 16, c2, nm2, acc);
+    if (UNSTEP_TURN_AT == 2 && turn_signal != 0u) mbar_arrive(turn_signal);
+    tc_wait_ld();
+    tmem_ld32(t_S + 96, h1);           // keys 96..127 again
+    tmem_st32(t_S, preg);              // P of keys 0..63 over score columns 0..31
+  }
+  {
+    uint32_t preg[32];
+    mask_block32<kMasked>(h0, 64, nvalid);
+    exp_block32(h0, preg, c2, nm2, acc);
+    if (UNSTEP_TURN_AT == 3 && turn_signal != 0u) mbar_arrive(turn_signal);
+    tc_wait_ld();
+    mask_block32<kMasked>(h1, 96, nvalid);
+    exp_block32(h1, preg + 16, c2, nm2, acc);
+    if (UNSTEP_TURN_AT == 4 && turn_signal != 0u) mbar_arrive(turn_signal);
+    tmem_st32(t_S + 32, preg);         // P of keys 64..127 over score columns 32..63
+    tc_wait_st();                      // both halves of P are in TMEM
+    tc_fence_before();
+    mbar_arrive(bar_p_half);
+    mbar_arrive(bar_p_half + 8);
+    TRACE(trace_role, trace_tile, 5);
+  }
+  {
+    const uint64_t t = add_f32x2(add_f32x2(acc[0], acc[1]), add_f32x2(acc[2], acc[3]));
+    float t0, t1;
+    unpack_f32x2(t, t0, t1);
+    l_run += t0 + t1;
+  }
+  return true;
+}
+
 __global__ void __launch_bounds__(kThreads, 1)
 window_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                    const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_kf,
@@ -411,9 +587,11 @@ window_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
   const uint32_t bar_s_full = sBar + 32 + 16 * kStages;      // [2]  MMA warp a -> softmax a
   const uint32_t bar_p_half = bar_s_full + 16;               // [2][2] softmax a -> MMA warp a
   const uint32_t bar_o_final = bar_p_half + 32;              // [2]  MMA warp a -> softmax a
-  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(gen + kSmemBar + 192);
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(gen + kSmemBar + 200);
-  volatile int* merge_flag = reinterpret_cast<volatile int*>(gen + kSmemBar + 208);
+  const uint32_t bar_turn = bar_o_final + 16;                // [2]  softmax 1-a -> softmax a: your turn on the MUFU pipe
+  const uint32_t bar_mturn = bar_turn + 16;                  // [2]  MMA warp 1-a -> MMA warp a: your turn on the tensor pipe
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(gen + kSmemBar + 224);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(gen + kSmemBar + 228);
+  volatile int* merge_flag = reinterpret_cast<volatile int*>(gen + kSmemBar + 232);   // [2]
   volatile float* xchg = reinterpret_cast<volatile float*>(gen + kSmemXchg);
 
   const int tid = threadIdx.x;
@@ -429,6 +607,8 @@ window_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
       mbar_init(bar_p_half + 16 * i, 128);
       mbar_init(bar_p_half + 16 * i + 8, 128);
       mbar_init(bar_o_final + 8 * i, 1);
+      mbar_init(bar_turn + 8 * i, 128);
+      mbar_init(bar_mturn + 8 * i, 1);
     }
     for (int i = 0; i < kStages; ++i) {
       mbar_init(bar_kv_full + 8 * i, 1);
@@ -500,7 +680,7 @@ window_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
       const int a = warp - 8;
       Sched sched(p);
       Seg s;
-      uint32_t kv_it = 0, q_it = 0, sp_it = 0;
+      uint32_t kv_it = 0, q_it = 0, sp_it = 0, mturn_it = 0;
       bool ok = true;
       const uint32_t idesc_pv = idesc_bf16_f32(kTileM, kHeadDim, 1);
       const uint32_t idesc_qk_full = idesc_bf16_f32(kTileM, kTileN, 0);
@@ -515,15 +695,16 @@ window_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
       auto issue_qk = [&](uint32_t stage, int valid) {
         const uint64_t dk = dk0 + static_cast<uint64_t>((stage * kTileBytes) >> 4);
         const uint32_t idesc = valid == kTileN ? idesc_qk_full : idesc_bf16_f32(kTileM, (valid + 15) & ~15, 0);
-#pragma unroll
-        for (int k = 0; k < 8; ++k) {
-          const uint64_t off = static_cast<uint64_t>(((k >> 2) * kHalfBytes + (k & 3) * 32) >> 4);
-          mma_ss(s_tmem, dq + off, dk + off, idesc, k > 0);
-        }
+        mma_ss_k128(s_tmem, dq, dk, idesc, 0u);
         tc_commit(my_s_full);
         tc_commit(bar_kv_empty + 8 * stage);
       };
       auto issue_pv_half = [&](uint64_t dv, int half, int k_steps, bool accumulate) {
+        if (k_steps >= 4 * half + 4) {
+          mma_ts_k64(o_tmem, s_tmem + 32 * half, dv + static_cast<uint64_t>(512 * half), idesc_pv,
+                     accumulate ? 1u : 0u);
+          return;
+        }
 #pragma unroll
         for (int k = 4 * half; k < 4 * half + 4; ++k)
           if (k < k_steps)
@@ -567,6 +748,24 @@ window_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
           if (part) {
             const uint64_t dv = dv0 + static_cast<uint64_t>((vst * kTileBytes) >> 4);
             TRACE(2 + a, sp_it, 0);
+#if UNSTEP_ROW_SOFTMAX
+            ok = w.spin(my_p_half, sp_it & 1);
+            if (!ok) break;
+            TRACE(2 + a, sp_it, 1);
+            ok = w.spin(my_p_half + 8, sp_it & 1);
+            if (!ok) break;
+            // The two issuers take turns with their P V + Q K^T chains: issued side by side the
+            // chains would interleave in the tensor pipe and finish together, which pulls the
+            // two query tiles into step; one after the other keeps them half a period apart.
+            if (s.nq == 2) {
+              ok = w.spin(bar_mturn + 8 * a, (a == 0) ? ((mturn_it & 1) ^ 1) : (mturn_it & 1));
+              if (!ok) break;
+            }
+            TRACE(2 + a, sp_it, 3);
+            tc_fence_after();
+            issue_pv_half(dv, 0, k_steps, j > 0);
+            issue_pv_half(dv, 1, k_steps, true);
+#else
             // both column halves of P (and any rescale of O) must be in before O is touched
             ok = w.wait(my_p_half, sp_it & 1);
             if (!ok) break;
@@ -577,10 +776,17 @@ window_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
             tc_fence_after();
             issue_pv_half(dv, 0, k_steps, j > 0);
             issue_pv_half(dv, 1, k_steps, true);
+#endif
             TRACE(2 + a, sp_it, 4);
             // the next S first (it is what the softmax warps wait for), the stage releases after it
             if (more) issue_qk(kst, valid);
             tc_commit(bar_kv_empty + 8 * vst);
+#if UNSTEP_ROW_SOFTMAX
+            if (s.nq == 2) {
+              mbar_arrive(bar_mturn + 8 * (1 - a));
+              ++mturn_it;
+            }
+#endif
             TRACE(2 + a, sp_it, 5);
             ++sp_it;
           } else {
@@ -596,6 +802,178 @@ window_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
       }
     }
   } else {
+#if UNSTEP_ROW_SOFTMAX
+    // ---------------------------------------------------------------- softmax warpgroups
+    // Warps 0-3 own query tile 0, warps 4-7 query tile 1; a thread owns a row from the scores
+    // to the output.  The groups never wait for each other.
+    reg_alloc_200();
+    const int a = warp >> 2;               // query tile of this warpgroup
+    const int row = tid & 127;             // row inside the tile = TMEM lane
+    const uint32_t t_lane = tmem_base + (static_cast<uint32_t>((warp & 3) * 32) << 16);
+    const uint32_t t_S = t_lane + a * 128, t_O = t_lane + 256 + a * 128;
+    const uint32_t my_p_half = bar_p_half + 16 * a;
+    volatile int* my_flag = merge_flag + a;
+    Sched sched(p);
+    Seg s;
+    uint32_t it = 0, seg_it = 0, pair_it = 0;
+    bool ok = true;
+    int seg_no = 0;
+    CTRACE(1);
+    // After a wait gave up (ok == false) a thread keeps walking its segments without working,
+    // so that it still meets its group at the barrier of the next split-item epilogue, where
+    // the whole group sees the abort flag and leaves together.
+    while (sched.next(s)) {
+      if (a >= s.nq) continue;             // a lone last query tile: nothing for group 1
+      float m_run = -INFINITY, l_run = 0.f;
+      const bool paired = (s.nq == 2);     // both groups walk this segment: take turns
+#ifdef UNSTEP_NO_EXP_TURN
+      const uint32_t turn_wait = 0u, turn_signal = 0u;
+#else
+      const uint32_t turn_wait = paired ? bar_turn + 8 * a : 0u;
+      const uint32_t turn_signal = paired ? bar_turn + 8 * (1 - a) : 0u;
+#endif
+      for (int j = s.t0; j < s.t1 && ok; ++j) {
+        const int valid = tile_info(p, s.b, j).valid;
+        TRACE(a, it, 0);
+        ok = w.wait(bar_s_full + 8 * a, it & 1);
+        if (!ok) break;
+        tc_fence_after();
+        if (it == 0) CTRACE(2);
+        TRACE(a, it, 1);
+        const uint32_t turn_parity = (a == 0) ? ((pair_it & 1) ^ 1) : (pair_it & 1);
+        if (valid < kTileN)
+          ok = softmax_row_tile<true>(t_S, t_O, p.scale_log2e, valid, j == s.t0, m_run, l_run, my_p_half, w,
+                                      turn_wait, turn_parity, turn_signal, a, it);
+        else
+          ok = softmax_row_tile<false>(t_S, t_O, p.scale_log2e, kTileN, j == s.t0, m_run, l_run, my_p_half, w,
+                                       turn_wait, turn_parity, turn_signal, a, it);
+        if (!ok) break;
+        ++it;
+        if (paired) ++pair_it;
+      }
+      CTRACE(8 + seg_no);
+      // ---- epilogue of this group's query tile ----
+      if (ok) {
+        ok = w.wait(bar_o_final + 8 * a, seg_it & 1);
+        ++seg_it;
+        tc_fence_after();
+      }
+      const int n = (2 * s.qp + a) * kTileM + row;
+      uint4* dst = reinterpret_cast<uint4*>(
+          out + ((static_cast<int64_t>(s.b) * p.L + n) * p.Hn + s.h) * kHeadDim);
+      auto store_row = [&](uint4* d, const float* v, float inv_l) {   // 32 columns
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          uint4 vv;
+          vv.x = pack_bf16x2(v[8 * i + 0] * inv_l, v[8 * i + 1] * inv_l);
+          vv.y = pack_bf16x2(v[8 * i + 2] * inv_l, v[8 * i + 3] * inv_l);
+          vv.z = pack_bf16x2(v[8 * i + 4] * inv_l, v[8 * i + 5] * inv_l);
+          vv.w = pack_bf16x2(v[8 * i + 6] * inv_l, v[8 * i + 7] * inv_l);
+          d[i] = vv;
+        }
+      };
+      const bool whole = (s.t0 == 0 && s.t1 == s.tiles);
+      if (whole) {
+        // O / l -> bf16 -> out[b][n][h][:]: a thread writes its whole 256-byte row
+        if (ok) {
+          const float inv_l = 1.f / l_run;
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            float o[32];
+            tmem_ld32(t_O + q * 32, reinterpret_cast<uint32_t*>(o));
+            tc_wait_ld();
+            if (n < p.L) store_row(dst + 4 * q, o, inv_l);
+          }
+        }
+      } else {
+        // Part of a split item.  The parts of an item's query tile are merged by whichever of
+        // them is done last, in part order (a fixed order, so the result does not depend on
+        // which one that is); the merging part takes its own accumulator straight from TMEM.
+        // A part that finds all others already published merges at once without publishing
+        // itself; otherwise it publishes (O, m, l), counts itself in, and merges if that made
+        // the count complete.
+        const int c_lo = Sched::cta_of(p, s.item_step0);
+        const int c_hi = Sched::cta_of(p, s.item_step0 + s.tiles - 1);
+        const int others = c_hi - c_lo;
+        int* counter = p.counters + 2 * s.item + a;
+        if (row == 0 && ok) {
+          int seen;
+          asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(seen) : "l"(counter) : "memory");
+          *my_flag = (seen == others) ? 1 : 0;
+        }
+        group_barrier(a);
+        if (*abort_flag) break;            // raised before the barrier by whoever gave up
+        bool last = (*my_flag != 0);
+        if (!last) {
+          float* mine = p.part + (static_cast<int64_t>(2 * blockIdx.x + (s.first_in_cta ? 0 : 1)) * kPartFloats +
+                                  a * kPartTileFloats);
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            uint32_t o[32];
+            tmem_ld32(t_O + q * 32, o);
+            tc_wait_ld();
+#pragma unroll
+            for (int i = 0; i < 32; ++i) mine[(q * 32 + i) * 128 + row] = __uint_as_float(o[i]);
+          }
+          mine[128 * 128 + row] = m_run;
+          mine[128 * 128 + 128 + row] = l_run;
+          __threadfence();
+          group_barrier(a);   // all of this part is published; everyone has read the flag
+          if (row == 0) *my_flag = (atomicAdd(counter, 1) == others) ? 1 : 0;
+          group_barrier(a);
+          last = (*my_flag != 0);
+        }
+        if (last) {
+          __threadfence();
+          if (row == 0) *counter = 0;   // ready for the next launch
+          const int me = static_cast<int>(blockIdx.x);
+          auto part_of = [&](int c) -> const float* {
+            const int64_t clo = Sched::cta_lo(p, c);
+            const bool first = clo >= s.item_step0;   // the part starts the range of CTA c
+            return p.part + (static_cast<int64_t>(2 * c + (first ? 0 : 1)) * kPartFloats + a * kPartTileFloats);
+          };
+          float m_all = m_run;
+          for (int c = c_lo; c <= c_hi; ++c)
+            if (c != me) m_all = fmaxf(m_all, __ldcg(part_of(c) + 128 * 128 + row));
+          float l_sum = 0.f;
+          for (int c = c_lo; c <= c_hi; ++c) {
+            const float* pc = part_of(c);
+            const float m_c = c == me ? m_run : __ldcg(pc + 128 * 128 + row);
+            const float l_c = c == me ? l_run : __ldcg(pc + 128 * 128 + 128 + row);
+            l_sum += l_c * ex2((m_c - m_all) * p.scale_log2e);
+          }
+          const float inv_l = 1.f / l_sum;
+#pragma unroll 1
+          for (int q = 0; q < 4; ++q) {   // 32 output columns at a time
+            float acc[32];
+#pragma unroll
+            for (int i = 0; i < 32; ++i) acc[i] = 0.f;
+            for (int c = c_lo; c <= c_hi; ++c) {
+              float v[32];
+              float m_c;
+              if (c == me) {
+                tmem_ld32(t_O + 32 * q, reinterpret_cast<uint32_t*>(v));
+                tc_wait_ld();
+                m_c = m_run;
+              } else {
+                const float* pc = part_of(c);
+#pragma unroll
+                for (int i = 0; i < 32; ++i) v[i] = __ldcg(pc + (32 * q + i) * 128 + row);
+                m_c = __ldcg(pc + 128 * 128 + row);
+              }
+              const float sc = ex2((m_c - m_all) * p.scale_log2e);
+#pragma unroll
+              for (int i = 0; i < 32; ++i) acc[i] = fmaf(v[i], sc, acc[i]);
+            }
+            if (n < p.L) store_row(dst + 4 * q, acc, inv_l);
+          }
+        }
+      }
+      tc_fence_before();
+      CTRACE(3 + seg_no);
+      ++seg_no;
+    }
+#else
     // ---------------------------------------------------------------- softmax warps
     reg_alloc_200();
     const int half = warp >> 2;            // which 64 key columns / output columns of the row
@@ -784,6 +1162,7 @@ window_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
       CTRACE(3 + seg_no);
       ++seg_no;
     }
+#endif
   }
 
   // ---- teardown: every role ends here, also after a timed-out wait --------------------
@@ -1063,7 +1442,7 @@ extern "C" int unstep_debug_read_cta_trace(unsigned long long* host_out) {
 }
 extern "C" int unstep_debug_read_trace(long long* host_out) {
   if (cudaDeviceSynchronize() != cudaSuccess) return UNSTEP_ERR_CUDA;
-  return cudaMemcpyFromSymbol(host_out, g_trace, sizeof(long long) * 4 * 64 * 8) == cudaSuccess
+  return cudaMemcpyFromSymbol(host_out, g_trace, sizeof(long long) * 12 * 64 * 8) == cudaSuccess
              ? UNSTEP_OK : UNSTEP_ERR_CUDA;
 }
 #endif
