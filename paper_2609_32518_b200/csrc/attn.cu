@@ -1,14 +1,16 @@
 // Windowed attention of one chunk over the KV ring (sm_100a).
 //
 // Persistent, warp-specialised kernel, one CTA per SM:
-//   warps 0-7   softmax: two threads per query row (64 key columns each); the eight warps
-//               work on one query tile at a time and alternate between the item's two tiles
+//   warps 0-3   softmax of query tile 0, one thread per query row
+//   warps 4-7   softmax of query tile 1
 //   warp  8, 9  tcgen05.mma issuers of query tile 0 and 1 (one lane each); warp 8 owns TMEM
 //   warp  10    TMA producer (one lane)
 // A work item is (stream, head, pair of 128-query tiles): both tiles share every K/V
-// tile, and the softmax of one overlaps the tensor-core work of the other.  S = Q K^T
-// and O += P V accumulate in TMEM; P (bf16) is written back over S and fed to the
-// second MMA straight from TMEM.
+// tile.  The two tiles run half a period apart: while one is in its exponentials (MUFU
+// pipe) the other's P V and next Q K^T run on the tensor core.  Two small token rings keep
+// them apart: the softmax groups take turns on the exponentials, the MMA issuers on the
+// tensor pipe.  S = Q K^T and O += P V accumulate in TMEM; P (bf16) is written back over S
+// and fed to the second MMA straight from TMEM.
 //
 // The attended frames are at most three runs of consecutive cache slots (sink prefix, ring
 // up to its end, ring from its start).  Key tiles are cut from the runs through a flat
@@ -75,8 +77,7 @@ constexpr float kRescaleThreshold = 8.f;    // log2 units: rescale O only when t
 constexpr int kSmemQ = 0;
 constexpr int kSmemKV = 2 * kTileBytes;
 constexpr int kSmemBar = kSmemKV + kStages * kTileBytes;
-constexpr int kSmemXchg = kSmemBar + 256;                // float[2][2][128]: row max / row sum exchange
-constexpr int kAttnSmemBytes = kSmemXchg + 2048;
+constexpr int kAttnSmemBytes = kSmemBar + 256;
 
 struct AttnParams {
   int32_t Hn, L, T, C;
@@ -226,34 +227,9 @@ struct Sched {
   }
 };
 
-__device__ __forceinline__ void named_barrier_128(int id) {
-  asm volatile("bar.sync %0, 128;" ::"r"(id) : "memory");
-}
-
 struct Waiter {
   volatile int* abort_flag;
   long long limit;   // clock cycles after which a wait gives up
-  // Bounded wait that polls without parking the thread: for the single-lane roles on the
-  // critical path of a tile, where the wake-up of a parked thread would add to every hand-over.
-  __device__ __forceinline__ bool spin(uint32_t bar, uint32_t parity) const {
-#ifdef UNSTEP_NO_SPIN
-    return wait(bar, parity);
-#else
-    if (mbar_test_wait(bar, parity)) return true;
-    const long long t0 = clock64();
-    for (uint32_t n = 1;; ++n) {
-      if (mbar_test_wait(bar, parity)) return true;
-      if ((n & 1023u) == 0u) {
-        if (*abort_flag) return false;
-        if (clock64() - t0 > limit) {
-          *abort_flag = 1;
-          atomicExch(&g_status, UNSTEP_ERR_TIMEOUT);
-          return false;
-        }
-      }
-    }
-#endif
-  }
   // Bounded wait: the hardware parks the thread between polls; the clock and the CTA's abort
   // flag are only looked at every 32 polls so that a waiting warp leaves the issue slots alone.
   __device__ __forceinline__ bool wait(uint32_t bar, uint32_t parity) const {
@@ -279,24 +255,6 @@ static_assert(128 * 96 + 256 * 200 <= 384 * 168, "register redistribution exceed
 __device__ __forceinline__ void reg_dealloc_96() { asm volatile("setmaxnreg.dec.sync.aligned.u32 96;"); }
 __device__ __forceinline__ void reg_alloc_200() { asm volatile("setmaxnreg.inc.sync.aligned.u32 200;"); }
 
-// --------------------------------------------------------------------------------------
-// Softmax of one 128 x 128 score tile.  All eight softmax warps work on the same tile: the
-// thread pair (warp w, warp w + 4) shares a query row, each taking 64 of its 128 key columns,
-// and the warps alternate between the two query tiles of the item.  So the exponentials of one
-// tile run on all four MUFU pipes at once, its P reaches the tensor core sooner, and while the
-// tensor core works on that tile the warps are busy with the other one.
-//   t_S / t_O : TMEM addresses (this warp's lanes) of the tile's scores and output
-//   half      : which 64 columns this thread owns
-//   xchg      : shared float[2][128] used to combine the two partial row maxima
-//   kMasked   : key columns >= nvalid are excluded (last tile of a frame)
-// The running maximum is only raised when it grows by more than 2^kRescaleThreshold, so the
-// output accumulator is rescaled rarely; P stays below 2^8 in between.  Both threads of a row
-// take the same decision from the same combined maximum.  The caller has seen S of this tile
-// complete, which (the tensor pipe runs in issue order) also means the previous P V into O has
-// landed, so O may be rescaled here without another wait.
-// P (bf16 pairs) overwrites the first 64 columns of S: this thread's 32 columns are written
-// only after the row's partner has loaded its scores (the barrier of the max exchange).
-// --------------------------------------------------------------------------------------
 // 2^x for a pair of floats without the MUFU pipe: x = n + f with n = round(x) (the add of
 // 1.5 * 2^23 leaves n in the low mantissa bits), 2^f by a cubic on [-0.5, 0.5] (relative error
 // 7.5e-5, far below the bf16 rounding of P), and n is added into the exponent field.
@@ -323,112 +281,14 @@ __device__ __forceinline__ void exp2_poly_pair(uint64_t x2, float& p0, float& p1
 #define UNSTEP_EMU_OF8 2   // of every 8 column pairs, this many take the polynomial instead of MUFU
 #endif
 
-__device__ __forceinline__ void softmax_barrier() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
-
-template <bool kMasked>
-__device__ __forceinline__ bool softmax_tile(uint32_t t_S, uint32_t t_O, float c, int nvalid,
-                                             bool first, int half, int row, volatile float* xchg,
-                                             volatile int* abort_flag, float& m_run, float& l_run,
-                                             uint32_t bar_p, int trace_role, int trace_tile) {
-  uint32_t sreg[64];
-  tmem_ld32(t_S + 64 * half, sreg);
-  tmem_ld32(t_S + 64 * half + 32, sreg + 32);
-  tc_wait_ld();
-  TRACE(trace_role, trace_tile, 2);
-  if (kMasked) {
-#pragma unroll
-    for (int i = 0; i < 64; ++i)
-      if (64 * half + i >= nvalid) sreg[i] = 0xFF800000u;  // -inf
-  }
-  // partial row maximum: two independent chains of 3-input max
-  float mx2[2];
-#pragma unroll
-  for (int q = 0; q < 2; ++q) {
-    float m = fmaxf(__uint_as_float(sreg[32 * q]), __uint_as_float(sreg[32 * q + 1]));
-#pragma unroll
-    for (int i = 2; i < 32; i += 2)
-      m = max3(m, __uint_as_float(sreg[32 * q + i]), __uint_as_float(sreg[32 * q + i + 1]));
-    mx2[q] = m;
-  }
-  float mx = fmaxf(mx2[0], mx2[1]);
-  xchg[half * 128 + row] = mx;
-  softmax_barrier();
-  // a thread whose wait gave up still comes to the barrier (nobody is left waiting there);
-  // the flag it raised before is visible to all now, and all leave together
-  if (*abort_flag) return false;
-  mx = fmaxf(mx, xchg[(1 - half) * 128 + row]);
-  TRACE(trace_role, trace_tile, 3);
-  float alpha = 1.f;
-  bool grow = false;
-  if (first) {
-    m_run = mx;
-  } else if ((mx - m_run) * c > kRescaleThreshold) {
-    alpha = ex2((m_run - mx) * c);
-    m_run = mx;
-    l_run *= alpha;
-    grow = true;
-  }
-  if (__any_sync(0xFFFFFFFFu, grow)) {
-#pragma unroll
-    for (int q = 0; q < 2; ++q) {
-      uint32_t o[32];
-      tmem_ld32(t_O + 64 * half + q * 32, o);
-      tc_wait_ld();
-#pragma unroll
-      for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
-      tmem_st32(t_O + 64 * half + q * 32, o);
-    }
-  }
-  // p = 2^(s*c - m*c): packed FMA on pairs, one MUFU per element, packed partial sums
-  const uint64_t c2 = pack_f32x2(c, c);
-  const float neg_ms = -m_run * c;
-  const uint64_t nm2 = pack_f32x2(neg_ms, neg_ms);
-  uint64_t acc[4] = {0ull, 0ull, 0ull, 0ull};
-  uint32_t preg[32];
-#pragma unroll
-  for (int i = 0; i < 32; ++i) {
-    const uint64_t x2 = fma_f32x2(pack_f32x2(__uint_as_float(sreg[2 * i]), __uint_as_float(sreg[2 * i + 1])),
-                                  c2, nm2);
-    float p0, p1;
-    if ((i & 7) < UNSTEP_EMU_OF8) {
-      // part of the exponentials runs on the FMA pipe: the MUFU pipe alone would bound the tile
-      exp2_poly_pair(x2, p0, p1);
-    } else {
-      float x0, x1;
-      unpack_f32x2(x2, x0, x1);
-      p0 = ex2(x0);
-      p1 = ex2(x1);
-    }
-    acc[i & 3] = add_f32x2(acc[i & 3], pack_f32x2(p0, p1));
-    preg[i] = pack_bf16x2(p0, p1);
-  }
-  tmem_st32(t_S + 32 * half, preg);
-  tc_wait_st();
-  tc_fence_before();
-  mbar_arrive(bar_p);
-  TRACE(trace_role, trace_tile, 4);
-  {
-    const uint64_t t = add_f32x2(add_f32x2(acc[0], acc[1]), add_f32x2(acc[2], acc[3]));
-    float t0, t1;
-    unpack_f32x2(t, t0, t1);
-    l_run += t0 + t1;
-  }
-  return true;
-}
-
-#ifndef UNSTEP_ROW_SOFTMAX
-#define UNSTEP_ROW_SOFTMAX 1
-#endif
-#ifndef UNSTEP_TURN_AT
-#define UNSTEP_TURN_AT 4
-#endif
 
 // --------------------------------------------------------------------------------------
 // Softmax of one 128 x 128 score tile with one thread per query row (a warpgroup per query
-// tile).  The two warpgroups run independently and drift half a period apart, so that one
-// is in its MUFU-bound exponentials while the other loads, reduces and stores, and the tensor
-// core works on one tile while the other is in its softmax.  No data crosses threads.
-// P is handed over in two halves of 64 keys, so P V can start on the first half.
+// tile); no data crosses threads.  The running maximum is only raised when it grows by more
+// than 2^kRescaleThreshold, so the output accumulator is rescaled rarely; P stays below 2^8 in
+// between.  The caller has seen S of this tile complete, which (the tensor pipe runs in issue
+// order) also means the previous P V into O has landed, so O may be rescaled here without
+// another wait.  Returns false when a bounded wait gave up.
 // --------------------------------------------------------------------------------------
 __device__ __forceinline__ void group_barrier(int a) {
   if (a == 0) asm volatile("bar.sync 1, 128;" ::: "memory");
@@ -477,7 +337,7 @@ __device__ __forceinline__ void mask_block32(uint32_t* s, int col0, int nvalid) 
 template <bool kMasked>
 __device__ __forceinline__ bool softmax_row_tile(uint32_t t_S, uint32_t t_O, float c, int nvalid,
                                                  bool first, float& m_run, float& l_run,
-                                                 uint32_t bar_p_half, const Waiter& w, uint32_t turn_wait,
+                                                 uint32_t bar_p_full, const Waiter& w, uint32_t turn_wait,
                                                  uint32_t turn_parity, uint32_t turn_signal,
                                                  int trace_role, int trace_tile) {
   uint32_t lo[64];
@@ -534,7 +394,6 @@ __device__ __forceinline__ bool softmax_row_tile(uint32_t t_S, uint32_t t_O, flo
     uint32_t preg[32];
     exp_block32(lo, preg, c2, nm2, acc);
     exp_block32(lo + 32, preg + 16, c2, nm2, acc);
-    if (UNSTEP_TURN_AT == 2 && turn_signal != 0u) mbar_arrive(turn_signal);
     tc_wait_ld();
     tmem_ld32(t_S + 96, h1);           // keys 96..127 again
     tmem_st32(t_S, preg);              // P of keys 0..63 over score columns 0..31
@@ -543,16 +402,14 @@ __device__ __forceinline__ bool softmax_row_tile(uint32_t t_S, uint32_t t_O, flo
     uint32_t preg[32];
     mask_block32<kMasked>(h0, 64, nvalid);
     exp_block32(h0, preg, c2, nm2, acc);
-    if (UNSTEP_TURN_AT == 3 && turn_signal != 0u) mbar_arrive(turn_signal);
     tc_wait_ld();
     mask_block32<kMasked>(h1, 96, nvalid);
     exp_block32(h1, preg + 16, c2, nm2, acc);
-    if (UNSTEP_TURN_AT == 4 && turn_signal != 0u) mbar_arrive(turn_signal);
+    if (turn_signal != 0u) mbar_arrive(turn_signal);   // the exponentials are done: the other group may go
     tmem_st32(t_S + 32, preg);         // P of keys 64..127 over score columns 32..63
     tc_wait_st();                      // both halves of P are in TMEM
     tc_fence_before();
-    mbar_arrive(bar_p_half);
-    mbar_arrive(bar_p_half + 8);
+    mbar_arrive(bar_p_full);
     TRACE(trace_role, trace_tile, 5);
   }
   {
@@ -585,14 +442,13 @@ window_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
   const uint32_t bar_kv_full = sBar + 32;                    // [kStages] TMA -> both MMA warps
   const uint32_t bar_kv_empty = sBar + 32 + 8 * kStages;     // [kStages] both MMA warps -> TMA
   const uint32_t bar_s_full = sBar + 32 + 16 * kStages;      // [2]  MMA warp a -> softmax a
-  const uint32_t bar_p_half = bar_s_full + 16;               // [2][2] softmax a -> MMA warp a
-  const uint32_t bar_o_final = bar_p_half + 32;              // [2]  MMA warp a -> softmax a
+  const uint32_t bar_p_full = bar_s_full + 16;               // [2]  softmax a -> MMA warp a (128 arrivals)
+  const uint32_t bar_o_final = bar_p_full + 16;              // [2]  MMA warp a -> softmax a
   const uint32_t bar_turn = bar_o_final + 16;                // [2]  softmax 1-a -> softmax a: your turn on the MUFU pipe
   const uint32_t bar_mturn = bar_turn + 16;                  // [2]  MMA warp 1-a -> MMA warp a: your turn on the tensor pipe
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(gen + kSmemBar + 224);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(gen + kSmemBar + 228);
   volatile int* merge_flag = reinterpret_cast<volatile int*>(gen + kSmemBar + 232);   // [2]
-  volatile float* xchg = reinterpret_cast<volatile float*>(gen + kSmemXchg);
 
   const int tid = threadIdx.x;
   const int warp = tid >> 5;
@@ -604,8 +460,7 @@ window_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
       mbar_init(bar_q_full + 8 * i, 1);
       mbar_init(bar_q_empty + 8 * i, 1);
       mbar_init(bar_s_full + 8 * i, 1);
-      mbar_init(bar_p_half + 16 * i, 128);
-      mbar_init(bar_p_half + 16 * i + 8, 128);
+      mbar_init(bar_p_full + 8 * i, 128);
       mbar_init(bar_o_final + 8 * i, 1);
       mbar_init(bar_turn + 8 * i, 128);
       mbar_init(bar_mturn + 8 * i, 1);
@@ -689,7 +544,7 @@ window_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
       const uint64_t dk0 = smem_desc_sw128(sKV, 16, 1024);                  // stage 0 as a K tile
       const uint64_t dv0 = smem_desc_sw128(sKV, kHalfBytes, 1024);          // stage 0 as a V tile (MN-major)
       const uint32_t s_tmem = tmem_base + a * 128, o_tmem = tmem_base + 256 + a * 128;
-      const uint32_t my_s_full = bar_s_full + 8 * a, my_p_half = bar_p_half + 16 * a;
+      const uint32_t my_s_full = bar_s_full + 8 * a, my_p_full = bar_p_full + 8 * a;
 
       // a ragged tile runs with N (for Q K^T) and K (for P V) rounded up to 16 keys
       auto issue_qk = [&](uint32_t stage, int valid) {
@@ -748,45 +603,28 @@ window_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
           if (part) {
             const uint64_t dv = dv0 + static_cast<uint64_t>((vst * kTileBytes) >> 4);
             TRACE(2 + a, sp_it, 0);
-#if UNSTEP_ROW_SOFTMAX
-            ok = w.spin(my_p_half, sp_it & 1);
+            ok = w.wait(my_p_full, sp_it & 1);   // P of this tile is in TMEM, O rescaled if need be
             if (!ok) break;
             TRACE(2 + a, sp_it, 1);
-            ok = w.spin(my_p_half + 8, sp_it & 1);
-            if (!ok) break;
             // The two issuers take turns with their P V + Q K^T chains: issued side by side the
             // chains would interleave in the tensor pipe and finish together, which pulls the
             // two query tiles into step; one after the other keeps them half a period apart.
             if (s.nq == 2) {
-              ok = w.spin(bar_mturn + 8 * a, (a == 0) ? ((mturn_it & 1) ^ 1) : (mturn_it & 1));
+              ok = w.wait(bar_mturn + 8 * a, (a == 0) ? ((mturn_it & 1) ^ 1) : (mturn_it & 1));
               if (!ok) break;
             }
             TRACE(2 + a, sp_it, 3);
             tc_fence_after();
             issue_pv_half(dv, 0, k_steps, j > 0);
             issue_pv_half(dv, 1, k_steps, true);
-#else
-            // both column halves of P (and any rescale of O) must be in before O is touched
-            ok = w.wait(my_p_half, sp_it & 1);
-            if (!ok) break;
-            TRACE(2 + a, sp_it, 1);
-            ok = w.wait(my_p_half + 8, sp_it & 1);
-            if (!ok) break;
-            TRACE(2 + a, sp_it, 3);
-            tc_fence_after();
-            issue_pv_half(dv, 0, k_steps, j > 0);
-            issue_pv_half(dv, 1, k_steps, true);
-#endif
             TRACE(2 + a, sp_it, 4);
             // the next S first (it is what the softmax warps wait for), the stage releases after it
             if (more) issue_qk(kst, valid);
             tc_commit(bar_kv_empty + 8 * vst);
-#if UNSTEP_ROW_SOFTMAX
             if (s.nq == 2) {
               mbar_arrive(bar_mturn + 8 * (1 - a));
               ++mturn_it;
             }
-#endif
             TRACE(2 + a, sp_it, 5);
             ++sp_it;
           } else {
@@ -802,7 +640,6 @@ window_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
       }
     }
   } else {
-#if UNSTEP_ROW_SOFTMAX
     // ---------------------------------------------------------------- softmax warpgroups
     // Warps 0-3 own query tile 0, warps 4-7 query tile 1; a thread owns a row from the scores
     // to the output.  The groups never wait for each other.
@@ -811,7 +648,7 @@ window_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
     const int row = tid & 127;             // row inside the tile = TMEM lane
     const uint32_t t_lane = tmem_base + (static_cast<uint32_t>((warp & 3) * 32) << 16);
     const uint32_t t_S = t_lane + a * 128, t_O = t_lane + 256 + a * 128;
-    const uint32_t my_p_half = bar_p_half + 16 * a;
+    const uint32_t my_p_full = bar_p_full + 8 * a;
     volatile int* my_flag = merge_flag + a;
     Sched sched(p);
     Seg s;
@@ -826,12 +663,8 @@ window_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
       if (a >= s.nq) continue;             // a lone last query tile: nothing for group 1
       float m_run = -INFINITY, l_run = 0.f;
       const bool paired = (s.nq == 2);     // both groups walk this segment: take turns
-#ifdef UNSTEP_NO_EXP_TURN
-      const uint32_t turn_wait = 0u, turn_signal = 0u;
-#else
       const uint32_t turn_wait = paired ? bar_turn + 8 * a : 0u;
       const uint32_t turn_signal = paired ? bar_turn + 8 * (1 - a) : 0u;
-#endif
       for (int j = s.t0; j < s.t1 && ok; ++j) {
         const int valid = tile_info(p, s.b, j).valid;
         TRACE(a, it, 0);
@@ -842,10 +675,10 @@ window_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         TRACE(a, it, 1);
         const uint32_t turn_parity = (a == 0) ? ((pair_it & 1) ^ 1) : (pair_it & 1);
         if (valid < kTileN)
-          ok = softmax_row_tile<true>(t_S, t_O, p.scale_log2e, valid, j == s.t0, m_run, l_run, my_p_half, w,
+          ok = softmax_row_tile<true>(t_S, t_O, p.scale_log2e, valid, j == s.t0, m_run, l_run, my_p_full, w,
                                       turn_wait, turn_parity, turn_signal, a, it);
         else
-          ok = softmax_row_tile<false>(t_S, t_O, p.scale_log2e, kTileN, j == s.t0, m_run, l_run, my_p_half, w,
+          ok = softmax_row_tile<false>(t_S, t_O, p.scale_log2e, kTileN, j == s.t0, m_run, l_run, my_p_full, w,
                                        turn_wait, turn_parity, turn_signal, a, it);
         if (!ok) break;
         ++it;
@@ -973,196 +806,6 @@ window_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
       CTRACE(3 + seg_no);
       ++seg_no;
     }
-#else
-    // ---------------------------------------------------------------- softmax warps
-    reg_alloc_200();
-    const int half = warp >> 2;            // which 64 key columns / output columns of the row
-    const int row = tid & 127;             // row inside the tile = TMEM lane
-    const uint32_t t_lane = tmem_base + (static_cast<uint32_t>((warp & 3) * 32) << 16);
-    Sched sched(p);
-    Seg s;
-    uint32_t it[2] = {0, 0}, seg_it[2] = {0, 0}, x_it = 0;
-    bool ok = true;
-    int seg_no = 0;
-    CTRACE(1);
-    while (ok && sched.next(s)) {
-      float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};
-      for (int j = s.t0; j < s.t1 && ok; ++j) {
-        const int valid = tile_info(p, s.b, j).valid;
-        const bool tail = valid < kTileN;
-#pragma unroll
-        for (int a = 0; a < 2; ++a) {
-          if (a >= s.nq) break;
-          TRACE(a, it[a], 0);
-          w.wait(bar_s_full + 8 * a, it[a] & 1);  // on failure the flag is up: handled after the barrier
-          tc_fence_after();
-          if (it[0] == 0) CTRACE(2);
-          TRACE(a, it[a], 1);
-          volatile float* xc = xchg + (x_it & 1) * 256;
-          const uint32_t t_S = t_lane + a * 128, t_O = t_lane + 256 + a * 128;
-          const uint32_t bar_p = bar_p_half + 16 * a + 8 * half;
-          if (tail)
-            ok = softmax_tile<true>(t_S, t_O, p.scale_log2e, valid, j == s.t0, half, row, xc,
-                                    abort_flag, m_run[a], l_run[a], bar_p, a, it[a]);
-          else
-            ok = softmax_tile<false>(t_S, t_O, p.scale_log2e, kTileN, j == s.t0, half, row, xc,
-                                     abort_flag, m_run[a], l_run[a], bar_p, a, it[a]);
-          if (!ok) break;
-          ++it[a];
-          ++x_it;
-        }
-      }
-      if (!ok) break;
-      CTRACE(8 + seg_no);
-      // ---- epilogue of the segment: both query tiles' accumulators are final ----
-      float l_all[2] = {0.f, 0.f};
-      for (int a = 0; a < s.nq; ++a) {
-        w.wait(bar_o_final + 8 * a, seg_it[a] & 1);
-        ++seg_it[a];
-        // row sum = the two partners' partial sums
-        volatile float* xc = xchg + (x_it & 1) * 256;
-        ++x_it;
-        xc[half * 128 + row] = l_run[a];
-        softmax_barrier();
-        if (*abort_flag) {
-          ok = false;
-          break;
-        }
-        l_all[a] = l_run[a] + xc[(1 - half) * 128 + row];
-      }
-      if (!ok) break;
-      tc_fence_after();
-      const bool whole = (s.t0 == 0 && s.t1 == s.tiles);
-      // this thread's 64 output columns of row n of query tile a
-      auto out_ptr = [&](int a) -> uint4* {
-        const int n = (2 * s.qp + a) * kTileM + row;
-        return reinterpret_cast<uint4*>(
-            out + ((static_cast<int64_t>(s.b) * p.L + n) * p.Hn + s.h) * kHeadDim + 64 * half);
-      };
-      auto store_row = [&](uint4* dst, const float* v, float inv_l) {   // 32 columns
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          uint4 vv;
-          vv.x = pack_bf16x2(v[8 * i + 0] * inv_l, v[8 * i + 1] * inv_l);
-          vv.y = pack_bf16x2(v[8 * i + 2] * inv_l, v[8 * i + 3] * inv_l);
-          vv.z = pack_bf16x2(v[8 * i + 4] * inv_l, v[8 * i + 5] * inv_l);
-          vv.w = pack_bf16x2(v[8 * i + 6] * inv_l, v[8 * i + 7] * inv_l);
-          dst[i] = vv;
-        }
-      };
-      if (whole) {
-        // O / l -> bf16 -> out[b][n][h][64*half ...]
-        for (int a = 0; a < s.nq; ++a) {
-          const uint32_t t_O = t_lane + 256 + a * 128 + 64 * half;
-          const bool in_range = (2 * s.qp + a) * kTileM + row < p.L;
-          const float inv_l = 1.f / l_all[a];
-          uint4* dst = out_ptr(a);
-#pragma unroll
-          for (int q = 0; q < 2; ++q) {
-            float o[32];
-            tmem_ld32(t_O + q * 32, reinterpret_cast<uint32_t*>(o));
-            tc_wait_ld();
-            if (in_range) store_row(dst + 4 * q, o, inv_l);
-          }
-        }
-      } else {
-        // Part of a split item.  The parts of an item are merged by whichever of them is done
-        // last, in part order (a fixed order, so the result does not depend on which one that
-        // is); the merging part takes its own accumulators straight from TMEM.  A part that
-        // finds all others already published merges at once without publishing itself;
-        // otherwise it publishes (O, m, l) of both tiles, counts itself in, and merges if
-        // that made the count complete.
-        const int c_lo = Sched::cta_of(p, s.item_step0);
-        const int c_hi = Sched::cta_of(p, s.item_step0 + s.tiles - 1);
-        const int others = c_hi - c_lo;
-        int* counter = p.counters + 2 * s.item;
-        if (tid == 0) {
-          int seen;
-          asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(seen) : "l"(counter) : "memory");
-          *merge_flag = (seen == others) ? 1 : 0;
-        }
-        softmax_barrier();
-        bool last = (*merge_flag != 0);
-        if (!last) {
-          float* mine = p.part + static_cast<int64_t>(2 * blockIdx.x + (s.first_in_cta ? 0 : 1)) * kPartFloats;
-          for (int a = 0; a < s.nq; ++a) {
-            const uint32_t t_O = t_lane + 256 + a * 128 + 64 * half;
-            float* dstp = mine + a * kPartTileFloats;
-#pragma unroll
-            for (int q = 0; q < 2; ++q) {
-              uint32_t o[32];
-              tmem_ld32(t_O + q * 32, o);
-              tc_wait_ld();
-#pragma unroll
-              for (int i = 0; i < 32; ++i) dstp[(64 * half + q * 32 + i) * 128 + row] = __uint_as_float(o[i]);
-            }
-            if (half == 0) {
-              dstp[128 * 128 + row] = m_run[a];
-              dstp[128 * 128 + 128 + row] = l_all[a];
-            }
-          }
-          __threadfence();
-          softmax_barrier();   // all of this part is published; everyone has read the flag
-          if (tid == 0) *merge_flag = (atomicAdd(counter, 1) == others) ? 1 : 0;
-          softmax_barrier();
-          last = (*merge_flag != 0);
-        }
-        if (last) {
-          __threadfence();
-          if (tid == 0) *counter = 0;   // ready for the next launch
-          const int me = static_cast<int>(blockIdx.x);
-          for (int a = 0; a < s.nq; ++a) {
-            auto part_of = [&](int c) -> const float* {
-              const int64_t clo = Sched::cta_lo(p, c);
-              const bool first = clo >= s.item_step0;   // the part starts the range of CTA c
-              return p.part + (static_cast<int64_t>(2 * c + (first ? 0 : 1)) * kPartFloats + a * kPartTileFloats);
-            };
-            const uint32_t t_O = t_lane + 256 + a * 128 + 64 * half;
-            float m_all = m_run[a];
-            for (int c = c_lo; c <= c_hi; ++c)
-              if (c != me) m_all = fmaxf(m_all, __ldcg(part_of(c) + 128 * 128 + row));
-            float l_sum = 0.f;
-            for (int c = c_lo; c <= c_hi; ++c) {
-              const float* pc = part_of(c);
-              const float m_c = c == me ? m_run[a] : __ldcg(pc + 128 * 128 + row);
-              const float l_c = c == me ? l_all[a] : __ldcg(pc + 128 * 128 + 128 + row);
-              l_sum += l_c * ex2((m_c - m_all) * p.scale_log2e);
-            }
-            const float inv_l = 1.f / l_sum;
-            float acc[64];
-#pragma unroll
-            for (int i = 0; i < 64; ++i) acc[i] = 0.f;
-            for (int c = c_lo; c <= c_hi; ++c) {
-              float v[64];
-              float m_c;
-              if (c == me) {
-                tmem_ld32(t_O, reinterpret_cast<uint32_t*>(v));
-                tmem_ld32(t_O + 32, reinterpret_cast<uint32_t*>(v) + 32);
-                tc_wait_ld();
-                m_c = m_run[a];
-              } else {
-                const float* pc = part_of(c);
-#pragma unroll
-                for (int i = 0; i < 64; ++i) v[i] = __ldcg(pc + (64 * half + i) * 128 + row);
-                m_c = __ldcg(pc + 128 * 128 + row);
-              }
-              const float sc = ex2((m_c - m_all) * p.scale_log2e);
-#pragma unroll
-              for (int i = 0; i < 64; ++i) acc[i] = fmaf(v[i], sc, acc[i]);
-            }
-            if ((2 * s.qp + a) * kTileM + row < p.L) {
-              uint4* dst = out_ptr(a);
-              store_row(dst, acc, inv_l);
-              store_row(dst + 4, acc + 32, inv_l);
-            }
-          }
-        }
-      }
-      tc_fence_before();
-      CTRACE(3 + seg_no);
-      ++seg_no;
-    }
-#endif
   }
 
   // ---- teardown: every role ends here, also after a timed-out wait --------------------
