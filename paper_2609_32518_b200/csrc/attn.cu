@@ -381,11 +381,13 @@ __device__ __forceinline__ bool softmax_row_tile(uint32_t t_S, uint32_t t_O, flo
   // The two warpgroups take turns on the exponentials: the MUFU pipe is shared, and alternating
   // keeps the two query tiles half a period apart, so that the tensor pipe has one tile's MMAs
   // to run while the other tile is in its softmax.
+  float neg_ms = -m_run * c;
   if (turn_wait != 0u && !w.wait(turn_wait, turn_parity)) return false;
+  // the exponentials take this value "from" the wait, so that they cannot be scheduled ahead of it
+  asm volatile("" : "+f"(neg_ms)::"memory");
   TRACE(trace_role, trace_tile, 6);
   // p = 2^(s*c - m*c): packed FMA on pairs, MUFU or polynomial, packed partial sums
   const uint64_t c2 = pack_f32x2(c, c);
-  const float neg_ms = -m_run * c;
   const uint64_t nm2 = pack_f32x2(neg_ms, neg_ms);
   uint64_t acc[4] = {0ull, 0ull, 0ull, 0ull};
   uint32_t h0[32], h1[32];
@@ -405,8 +407,9 @@ __device__ __forceinline__ bool softmax_row_tile(uint32_t t_S, uint32_t t_O, flo
     tc_wait_ld();
     mask_block32<kMasked>(h1, 96, nvalid);
     exp_block32(h1, preg + 16, c2, nm2, acc);
-    if (turn_signal != 0u) mbar_arrive(turn_signal);   // the exponentials are done: the other group may go
     tmem_st32(t_S + 32, preg);         // P of keys 64..127 over score columns 32..63
+    // the exponentials are done (the store consumes the last of them): the other group may go
+    if (turn_signal != 0u) mbar_arrive(turn_signal);
     tc_wait_st();                      // both halves of P are in TMEM
     tc_fence_before();
     mbar_arrive(bar_p_full);
