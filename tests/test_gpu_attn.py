@@ -139,3 +139,28 @@ def test_queries_shorter_than_a_tile_and_single_head():
     wl = W.Workload("short", sh, seed=25, history_starts=((0, 2, 4), (0,)), measured_starts=(6, 2),
                     window_frames=(6, 3, 2), k_scale=4.0)
     run(wl)
+
+
+def test_split_items_merge_in_a_fixed_order_bitwise_repeatable():
+    # The 1.3B shape leaves 80 of its 228 work items to be split along the keys between CTAs;
+    # whichever part finishes last merges them, in part order, so repeated launches must agree
+    # bit for bit although the finishing order varies.  A large K scale forces rescales of O.
+    wl = W.WORKLOADS["cfg3"]
+    sh = wl.shape
+    gen = torch.Generator(device="cuda").manual_seed(5)
+    dims = (sh.batch, sh.ring_frames, sh.tokens_per_frame, sh.heads, sh.head_dim)
+    ring_k = (4.0 * torch.randn(dims, generator=gen, device="cuda")).to(torch.bfloat16)
+    ring_v = torch.randn(dims, generator=gen, device="cuda").to(torch.bfloat16)
+    q = torch.randn((sh.batch, sh.chunk_tokens, sh.heads, sh.head_dim), generator=gen,
+                    device="cuda").to(torch.bfloat16)
+    abi = U.Shape.make(sh.batch, sh.heads, sh.chunk_frames, sh.grid_h, sh.grid_w, sh.ring_frames)
+    for wf in (21, 6):
+        outs = []
+        for _ in range(4):
+            out = torch.empty_like(q)
+            U.window_attn(abi, [42], wf, q, ring_k, ring_v, out)
+            outs.append(out.view(torch.int16).clone())
+        torch.cuda.synchronize()
+        assert all(torch.equal(outs[0], o) for o in outs[1:]), f"Wf={wf}: launches differ"
+        assert torch.isfinite(out.float()).all()
+    assert U.poll_status() == 0
