@@ -72,7 +72,6 @@ constexpr int kStages = 5;                  // 32 KB buffers shared by the K and
 constexpr int kThreads = 384;
 constexpr int kTmemCols = 512;              // S0 | S1 | O0 | O1, 128 fp32 columns each
 constexpr long long kWaitCycles = 2000000000LL;  // about a second: then give up, never hang
-constexpr float kRescaleThreshold = 8.f;    // log2 units: rescale O only when the max grows by 2^8
 
 constexpr int kSmemQ = 0;
 constexpr int kSmemKV = 2 * kTileBytes;
@@ -330,10 +329,62 @@ __device__ __forceinline__ void mask_block32(uint32_t* s, int col0, int nvalid) 
   }
 }
 
-// The scores are read from TMEM twice to keep the register count down: a first pass for the
-// row maximum (keys 64..127, then 0..63, the latter kept), then the exponentials of keys 0..63
-// from registers while keys 64..127 are fetched again in two blocks of 32.  P (bf16 pairs)
-// overwrites score columns 0..63, which are in registers by then.
+// Exponentials of the 128 scores of a row (TMEM columns t_S .. t_S + 127) against the reference
+// maximum m_run: keys 0..63 come in through `lo` (already in registers when lo_loaded), keys
+// 64..127 are fetched in two blocks of 32 while the first half is exponentiated.  Leaves P
+// (bf16 pairs) in p0 (keys 0..63) and p1 (keys 64..127) and returns the row's sum of P.
+template <bool kMasked>
+__device__ __forceinline__ float exp_row(uint32_t t_S, const uint32_t* lo, float c, float neg_ms, int nvalid,
+                                         uint32_t* p0, uint32_t* p1) {
+  const uint64_t c2 = pack_f32x2(c, c);
+  const uint64_t nm2 = pack_f32x2(neg_ms, neg_ms);
+  uint64_t acc[4] = {0ull, 0ull, 0ull, 0ull};
+  uint32_t h0[32], h1[32];
+  tmem_ld32(t_S + 64, h0);             // keys 64..95, in flight during the first half
+  exp_block32(lo, p0, c2, nm2, acc);
+  exp_block32(lo + 32, p0 + 16, c2, nm2, acc);
+  tc_wait_ld();
+  tmem_ld32(t_S + 96, h1);             // keys 96..127
+  mask_block32<kMasked>(h0, 64, nvalid);
+  exp_block32(h0, p1, c2, nm2, acc);
+  tc_wait_ld();
+  mask_block32<kMasked>(h1, 96, nvalid);
+  exp_block32(h1, p1 + 16, c2, nm2, acc);
+  const uint64_t t = add_f32x2(add_f32x2(acc[0], acc[1]), add_f32x2(acc[2], acc[3]));
+  float t0, t1;
+  unpack_f32x2(t, t0, t1);
+  return t0 + t1;
+}
+
+// Row maximum of the 128 scores in TMEM; leaves keys 0..63 (masked) in `lo`.
+template <bool kMasked>
+__device__ __forceinline__ float max_row(uint32_t t_S, uint32_t* lo, int nvalid) {
+  uint32_t hi[64];
+  tmem_ld32(t_S + 64, hi);
+  tmem_ld32(t_S + 96, hi + 32);
+  tmem_ld32(t_S, lo);
+  tmem_ld32(t_S + 32, lo + 32);
+  tc_wait_ld();
+  mask_block32<kMasked>(hi, 64, nvalid);
+  mask_block32<kMasked>(hi + 32, 96, nvalid);
+  mask_block32<kMasked>(lo, 0, nvalid);
+  mask_block32<kMasked>(lo + 32, 32, nvalid);
+  return fmaxf(fmaxf(max_block32(hi), max_block32(hi + 32)), fmaxf(max_block32(lo), max_block32(lo + 32)));
+}
+
+// Only the first key tile of a segment looks for the row maximum before its exponentials.
+// Every later tile exponentiates against that reference straight away and looks at the row's sum
+// of P afterwards.  P is positive, so a sum of at most kOptimisticLimit = 2^64 means that no
+// score was more than 64 (log2 units) above the reference: P (bf16) and the float32 sums are as
+// accurate at that magnitude as near 1 (same relative precision, no overflow: 128 keys of 2^64
+// times |v| stay far below 2^127), and everything accumulated before such a jump is negligible
+// exactly as in the true softmax.  Otherwise (scores more than 64 above the first tile's maximum,
+// or an overflow to inf) the warp finds the tile's true maximum, rescales O and l, and redoes
+// the exponentials; the scores are still in TMEM, because P is only stored at the very end.
+// Scores are read from TMEM in blocks to keep the register count down; P (bf16 pairs)
+// overwrites score columns 0..63.
+constexpr float kOptimisticLimit = 18446744073709551616.f;   // 2^64
+
 template <bool kMasked>
 __device__ __forceinline__ bool softmax_row_tile(uint32_t t_S, uint32_t t_O, float c, int nvalid,
                                                  bool first, float& m_run, float& l_run,
@@ -341,33 +392,35 @@ __device__ __forceinline__ bool softmax_row_tile(uint32_t t_S, uint32_t t_O, flo
                                                  uint32_t turn_parity, uint32_t turn_signal,
                                                  int trace_role, int trace_tile) {
   uint32_t lo[64];
-  float mx;
-  {
-    uint32_t hi[64];
-    tmem_ld32(t_S + 64, hi);
-    tmem_ld32(t_S + 96, hi + 32);
+  if (first) {
+    m_run = max_row<kMasked>(t_S, lo, nvalid);
+  } else {
     tmem_ld32(t_S, lo);
     tmem_ld32(t_S + 32, lo + 32);
     tc_wait_ld();
-    TRACE(trace_role, trace_tile, 2);
-    mask_block32<kMasked>(hi, 64, nvalid);
-    mask_block32<kMasked>(hi + 32, 96, nvalid);
     mask_block32<kMasked>(lo, 0, nvalid);
     mask_block32<kMasked>(lo + 32, 32, nvalid);
-    mx = fmaxf(fmaxf(max_block32(hi), max_block32(hi + 32)), fmaxf(max_block32(lo), max_block32(lo + 32)));
   }
-  TRACE(trace_role, trace_tile, 3);
-  float alpha = 1.f;
-  bool grow = false;
-  if (first) {
-    m_run = mx;
-  } else if ((mx - m_run) * c > kRescaleThreshold) {
-    alpha = ex2((m_run - mx) * c);
-    m_run = mx;
-    l_run *= alpha;
-    grow = true;
-  }
-  if (__any_sync(0xFFFFFFFFu, grow)) {
+  TRACE(trace_role, trace_tile, 2);
+  // The two warpgroups take turns on the exponentials: the MUFU pipe is shared, and alternating
+  // keeps the two query tiles half a period apart, so that the tensor pipe has one tile's MMAs
+  // to run while the other tile is in its softmax.
+  float neg_ms = -m_run * c;
+  if (turn_wait != 0u && !w.wait(turn_wait, turn_parity)) return false;
+  // the exponentials take this value "from" the wait, so that they cannot be scheduled ahead of it
+  asm volatile("" : "+f"(neg_ms)::"memory");
+  TRACE(trace_role, trace_tile, 6);
+  uint32_t p0[32], p1[32];
+  float sum = exp_row<kMasked>(t_S, lo, c, neg_ms, nvalid, p0, p1);
+  const bool redo = !first && !(sum <= kOptimisticLimit);   // also taken for inf and NaN
+  if (__any_sync(0xFFFFFFFFu, redo)) {
+    const float mx = max_row<kMasked>(t_S, lo, nvalid);
+    float alpha = 1.f;
+    if (mx > m_run) {
+      alpha = ex2((m_run - mx) * c);
+      m_run = mx;
+      l_run *= alpha;
+    }
 #pragma unroll
     for (int q = 0; q < 4; ++q) {
       uint32_t o[32];
@@ -377,50 +430,17 @@ __device__ __forceinline__ bool softmax_row_tile(uint32_t t_S, uint32_t t_O, flo
       for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
       tmem_st32(t_O + q * 32, o);
     }
+    sum = exp_row<kMasked>(t_S, lo, c, -m_run * c, nvalid, p0, p1);
   }
-  // The two warpgroups take turns on the exponentials: the MUFU pipe is shared, and alternating
-  // keeps the two query tiles half a period apart, so that the tensor pipe has one tile's MMAs
-  // to run while the other tile is in its softmax.
-  float neg_ms = -m_run * c;
-  if (turn_wait != 0u && !w.wait(turn_wait, turn_parity)) return false;
-  // the exponentials take this value "from" the wait, so that they cannot be scheduled ahead of it
-  asm volatile("" : "+f"(neg_ms)::"memory");
-  TRACE(trace_role, trace_tile, 6);
-  // p = 2^(s*c - m*c): packed FMA on pairs, MUFU or polynomial, packed partial sums
-  const uint64_t c2 = pack_f32x2(c, c);
-  const uint64_t nm2 = pack_f32x2(neg_ms, neg_ms);
-  uint64_t acc[4] = {0ull, 0ull, 0ull, 0ull};
-  uint32_t h0[32], h1[32];
-  tmem_ld32(t_S + 64, h0);             // keys 64..95 again, in flight during the first half
-  {
-    uint32_t preg[32];
-    exp_block32(lo, preg, c2, nm2, acc);
-    exp_block32(lo + 32, preg + 16, c2, nm2, acc);
-    tc_wait_ld();
-    tmem_ld32(t_S + 96, h1);           // keys 96..127 again
-    tmem_st32(t_S, preg);              // P of keys 0..63 over score columns 0..31
-  }
-  {
-    uint32_t preg[32];
-    mask_block32<kMasked>(h0, 64, nvalid);
-    exp_block32(h0, preg, c2, nm2, acc);
-    tc_wait_ld();
-    mask_block32<kMasked>(h1, 96, nvalid);
-    exp_block32(h1, preg + 16, c2, nm2, acc);
-    tmem_st32(t_S + 32, preg);         // P of keys 64..127 over score columns 32..63
-    // the exponentials are done (the store consumes the last of them): the other group may go
-    if (turn_signal != 0u) mbar_arrive(turn_signal);
-    tc_wait_st();                      // both halves of P are in TMEM
-    tc_fence_before();
-    mbar_arrive(bar_p_full);
-    TRACE(trace_role, trace_tile, 5);
-  }
-  {
-    const uint64_t t = add_f32x2(add_f32x2(acc[0], acc[1]), add_f32x2(acc[2], acc[3]));
-    float t0, t1;
-    unpack_f32x2(t, t0, t1);
-    l_run += t0 + t1;
-  }
+  tmem_st32(t_S, p0);        // P of keys 0..63 over score columns 0..31
+  tmem_st32(t_S + 32, p1);   // P of keys 64..127 over score columns 32..63
+  // the exponentials are done (the stores consume the last of them): the other group may go
+  if (turn_signal != 0u) mbar_arrive(turn_signal);
+  tc_wait_st();
+  tc_fence_before();
+  mbar_arrive(bar_p_full);
+  TRACE(trace_role, trace_tile, 5);
+  l_run += sum;
   return true;
 }
 

@@ -164,3 +164,21 @@ def test_split_items_merge_in_a_fixed_order_bitwise_repeatable():
         assert all(torch.equal(outs[0], o) for o in outs[1:]), f"Wf={wf}: launches differ"
         assert torch.isfinite(out.float()).all()
     assert U.poll_status() == 0
+
+
+def test_scores_far_above_the_first_tiles_maximum_take_the_redo_path():
+    # Later key tiles are exponentiated against the first tile's row maximum and only checked
+    # afterwards; scores more than 64 (log2 units) above it make the kernel find the true
+    # maximum, rescale and redo the tile.  History with ordinary keys, then a chunk whose keys are
+    # 64 times larger: its scores have a standard deviation of ~90 log2 units.
+    base = W.WORKLOADS["cfg1"]
+    dev, ora = DevicePath(base.shape), OraclePath(base.shape)
+    stream_history(base, dev, ora)
+    big = W.Workload("huge_keys", base.shape, seed=26, history_starts=base.history_starts,
+                     measured_starts=base.measured_starts, window_frames=(6, 4), k_scale=64.0)
+    run(big, dev=dev, ora=ora)
+    # and back to ordinary keys on top of the huge ones (the reference maximum is now far too high
+    # for most rows of the newest keys: their weights underflow, as in the exact softmax)
+    after = W.Workload("after_huge", base.shape, seed=27, history_starts=base.history_starts,
+                       measured_starts=(6,), window_frames=(6, 2))
+    run(after, dev=dev, ora=ora)
