@@ -257,11 +257,12 @@ __device__ __forceinline__ void reg_alloc_200() { asm volatile("setmaxnreg.inc.s
 // 2^x for a pair of floats without the MUFU pipe: x = n + f with n = round(x) (the add of
 // 1.5 * 2^23 leaves n in the low mantissa bits), 2^f by a cubic on [-0.5, 0.5] (relative error
 // 7.5e-5, far below the bf16 rounding of P), and n is added into the exponent field.
-// Inputs are clamped at -126 so that the exponent never wraps; -inf gives about 1e-38.
+// Inputs are clamped to [-126, 127] so that the exponent never wraps: -inf gives about 1e-38,
+// anything above 127 gives 2^127, which the caller's check of the row sum then catches.
 __device__ __forceinline__ void exp2_poly_pair(uint64_t x2, float& p0, float& p1) {
   float x0, x1;
   unpack_f32x2(x2, x0, x1);
-  const uint64_t xc = pack_f32x2(fmaxf(x0, -126.f), fmaxf(x1, -126.f));
+  const uint64_t xc = pack_f32x2(fminf(fmaxf(x0, -126.f), 127.f), fminf(fmaxf(x1, -126.f), 127.f));
   const uint64_t magic = pack_f32x2(12582912.f, 12582912.f);
   const uint64_t t2 = add_f32x2(xc, magic);
   const uint64_t n2 = add_f32x2(t2, pack_f32x2(-12582912.f, -12582912.f));

@@ -182,3 +182,24 @@ def test_scores_far_above_the_first_tiles_maximum_take_the_redo_path():
     after = W.Workload("after_huge", base.shape, seed=27, history_starts=base.history_starts,
                        measured_starts=(6,), window_frames=(6, 2))
     run(after, dev=dev, ora=ora)
+
+
+def test_single_huge_key_on_a_polynomial_column_is_caught():
+    # One key of a late tile, in a column whose exponential runs on the FMA pipe (the polynomial
+    # clamps its input, so an overflow there shows up as 2^127, not inf), scores hundreds of log2
+    # units above everything else for about half of the rows: those rows must still be redone.
+    wl = W.WORKLOADS["cfg1"]
+    dev, ora = DevicePath(wl.shape), OraclePath(wl.shape)
+    stream_history(wl, dev, ora)             # 4 frames of 64 tokens = two full key tiles
+    s = wl.measured_starts
+    q, k, v = W.batch_qkv(wl, s, 3)
+    k = k.copy()
+    k[:, 0] = W.f32_to_bf16_bits(W.bf16_bits_to_f32(k[:, 0]) * np.float32(256.0))   # column 0 of tile 2
+    q_dev = dev.append(s, q, k, v)
+    q_ref = ora.append(s, q, k, v)
+    assert np.array_equal(to_bits(q_dev), q_ref)
+    assert_ring_equal(dev, ora)
+    for wf in wl.window_frames:
+        out = to_bits(dev.attend(s, wf, q_dev))
+        check(out, ora.attend(s, wf, q_ref), f"huge key Wf={wf}")
+    assert U.poll_status() == 0
