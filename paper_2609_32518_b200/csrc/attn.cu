@@ -7,10 +7,10 @@
 //   warp  10    TMA producer (one lane)
 // A work item is (stream, head, pair of 128-query tiles): both tiles share every K/V
 // tile.  The two tiles run half a period apart: while one is in its exponentials (MUFU
-// pipe) the other's P V and next Q K^T run on the tensor core.  Two small token rings keep
-// them apart: the softmax groups take turns on the exponentials, the MMA issuers on the
-// tensor pipe.  S = Q K^T and O += P V accumulate in TMEM; P (bf16) is written back over S
-// and fed to the second MMA straight from TMEM.
+// pipe) the other's P V and next Q K^T run on the tensor core.  A small token ring keeps
+// them apart: the MMA issuers take turns on the tensor pipe.  S = Q K^T and O += P V
+// accumulate in TMEM; P (bf16) is written back over S and fed to the second MMA straight
+// from TMEM.
 //
 // The attended frames are at most three runs of consecutive cache slots (sink prefix, ring
 // up to its end, ring from its start).  Key tiles are cut from the runs through a flat
@@ -278,7 +278,7 @@ __device__ __forceinline__ void exp2_poly_pair(uint64_t x2, float& p0, float& p1
 }
 
 #ifndef UNSTEP_EMU_OF8
-#define UNSTEP_EMU_OF8 2   // of every 8 column pairs, this many take the polynomial instead of MUFU
+#define UNSTEP_EMU_OF8 0   // of every 8 column pairs, this many take the polynomial instead of MUFU
 #endif
 
 
@@ -288,7 +288,7 @@ __device__ __forceinline__ void exp2_poly_pair(uint64_t x2, float& p0, float& p1
 // than 2^kRescaleThreshold, so the output accumulator is rescaled rarely; P stays below 2^8 in
 // between.  The caller has seen S of this tile complete, which (the tensor pipe runs in issue
 // order) also means the previous P V into O has landed, so O may be rescaled here without
-// another wait.  Returns false when a bounded wait gave up.
+// another wait.
 // --------------------------------------------------------------------------------------
 __device__ __forceinline__ void group_barrier(int a) {
   if (a == 0) asm volatile("bar.sync 1, 128;" ::: "memory");
@@ -387,11 +387,9 @@ __device__ __forceinline__ float max_row(uint32_t t_S, uint32_t* lo, int nvalid)
 constexpr float kOptimisticLimit = 18446744073709551616.f;   // 2^64
 
 template <bool kMasked>
-__device__ __forceinline__ bool softmax_row_tile(uint32_t t_S, uint32_t t_O, float c, int nvalid,
+__device__ __forceinline__ void softmax_row_tile(uint32_t t_S, uint32_t t_O, float c, int nvalid,
                                                  bool first, float& m_run, float& l_run,
-                                                 uint32_t bar_p_full, const Waiter& w, uint32_t turn_wait,
-                                                 uint32_t turn_parity, uint32_t turn_signal,
-                                                 int trace_role, int trace_tile) {
+                                                 uint32_t bar_p_full, int trace_role, int trace_tile) {
   uint32_t lo[64];
   if (first) {
     m_run = max_row<kMasked>(t_S, lo, nvalid);
@@ -403,14 +401,7 @@ __device__ __forceinline__ bool softmax_row_tile(uint32_t t_S, uint32_t t_O, flo
     mask_block32<kMasked>(lo + 32, 32, nvalid);
   }
   TRACE(trace_role, trace_tile, 2);
-  // The two warpgroups take turns on the exponentials: the MUFU pipe is shared, and alternating
-  // keeps the two query tiles half a period apart, so that the tensor pipe has one tile's MMAs
-  // to run while the other tile is in its softmax.
-  float neg_ms = -m_run * c;
-  if (turn_wait != 0u && !w.wait(turn_wait, turn_parity)) return false;
-  // the exponentials take this value "from" the wait, so that they cannot be scheduled ahead of it
-  asm volatile("" : "+f"(neg_ms)::"memory");
-  TRACE(trace_role, trace_tile, 6);
+  const float neg_ms = -m_run * c;
   uint32_t p0[32], p1[32];
   float sum = exp_row<kMasked>(t_S, lo, c, neg_ms, nvalid, p0, p1);
   const bool redo = !first && !(sum <= kOptimisticLimit);   // also taken for inf and NaN
@@ -435,14 +426,11 @@ __device__ __forceinline__ bool softmax_row_tile(uint32_t t_S, uint32_t t_O, flo
   }
   tmem_st32(t_S, p0);        // P of keys 0..63 over score columns 0..31
   tmem_st32(t_S + 32, p1);   // P of keys 64..127 over score columns 32..63
-  // the exponentials are done (the stores consume the last of them): the other group may go
-  if (turn_signal != 0u) mbar_arrive(turn_signal);
   tc_wait_st();
   tc_fence_before();
   mbar_arrive(bar_p_full);
   TRACE(trace_role, trace_tile, 5);
   l_run += sum;
-  return true;
 }
 
 __global__ void __launch_bounds__(kThreads, 1)
@@ -468,8 +456,7 @@ window_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
   const uint32_t bar_s_full = sBar + 32 + 16 * kStages;      // [2]  MMA warp a -> softmax a
   const uint32_t bar_p_full = bar_s_full + 16;               // [2]  softmax a -> MMA warp a (128 arrivals)
   const uint32_t bar_o_final = bar_p_full + 16;              // [2]  MMA warp a -> softmax a
-  const uint32_t bar_turn = bar_o_final + 16;                // [2]  softmax 1-a -> softmax a: your turn on the MUFU pipe
-  const uint32_t bar_mturn = bar_turn + 16;                  // [2]  MMA warp 1-a -> MMA warp a: your turn on the tensor pipe
+  const uint32_t bar_mturn = bar_o_final + 16;                 // [2]  MMA warp 1-a -> MMA warp a: your turn on the tensor pipe
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(gen + kSmemBar + 224);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(gen + kSmemBar + 228);
   volatile int* merge_flag = reinterpret_cast<volatile int*>(gen + kSmemBar + 232);   // [2]
@@ -486,7 +473,6 @@ window_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
       mbar_init(bar_s_full + 8 * i, 1);
       mbar_init(bar_p_full + 8 * i, 128);
       mbar_init(bar_o_final + 8 * i, 1);
-      mbar_init(bar_turn + 8 * i, 128);
       mbar_init(bar_mturn + 8 * i, 1);
     }
     for (int i = 0; i < kStages; ++i) {
@@ -676,7 +662,7 @@ window_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
     volatile int* my_flag = merge_flag + a;
     Sched sched(p);
     Seg s;
-    uint32_t it = 0, seg_it = 0, pair_it = 0;
+    uint32_t it = 0, seg_it = 0;
     bool ok = true;
     int seg_no = 0;
     CTRACE(1);
@@ -686,9 +672,6 @@ window_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
     while (sched.next(s)) {
       if (a >= s.nq) continue;             // a lone last query tile: nothing for group 1
       float m_run = -INFINITY, l_run = 0.f;
-      const bool paired = (s.nq == 2);     // both groups walk this segment: take turns
-      const uint32_t turn_wait = paired ? bar_turn + 8 * a : 0u;
-      const uint32_t turn_signal = paired ? bar_turn + 8 * (1 - a) : 0u;
       for (int j = s.t0; j < s.t1 && ok; ++j) {
         const int valid = tile_info(p, s.b, j).valid;
         TRACE(a, it, 0);
@@ -697,16 +680,11 @@ window_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         tc_fence_after();
         if (it == 0) CTRACE(2);
         TRACE(a, it, 1);
-        const uint32_t turn_parity = (a == 0) ? ((pair_it & 1) ^ 1) : (pair_it & 1);
         if (valid < kTileN)
-          ok = softmax_row_tile<true>(t_S, t_O, p.scale_log2e, valid, j == s.t0, m_run, l_run, my_p_full, w,
-                                      turn_wait, turn_parity, turn_signal, a, it);
+          softmax_row_tile<true>(t_S, t_O, p.scale_log2e, valid, j == s.t0, m_run, l_run, my_p_full, a, it);
         else
-          ok = softmax_row_tile<false>(t_S, t_O, p.scale_log2e, kTileN, j == s.t0, m_run, l_run, my_p_full, w,
-                                       turn_wait, turn_parity, turn_signal, a, it);
-        if (!ok) break;
+          softmax_row_tile<false>(t_S, t_O, p.scale_log2e, kTileN, j == s.t0, m_run, l_run, my_p_full, a, it);
         ++it;
-        if (paired) ++pair_it;
       }
       CTRACE(8 + seg_no);
       // ---- epilogue of this group's query tile ----
