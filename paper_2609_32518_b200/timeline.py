@@ -6,7 +6,7 @@ shape and prints, for CTA 0, the clock64 stamps that the kernel's roles leave pe
 
   softmax warps (one line per warp 0..3 of each query tile's group):
       wait = starts waiting for S, s_rdy = S complete, ld = first scores in registers,
-      p = P handed to the tensor core, turn = its turn on the MUFU pipe
+      p = P handed to the tensor core
   MMA issuers: wait_p = starts waiting for P, got_p = P arrived, got_turn = its turn on the
       tensor pipe, pv = P V issued, qk = next Q K^T issued and committed
 
@@ -82,8 +82,8 @@ def main():
     print(f"workload {args.workload}, window {wf} frames, CTA 0, key tiles {lo}..{hi - 1}; cycles since tile {lo}")
     for a in (0, 1):
         for w in range(4):
-            print(f"softmax group {a} warp {w}: [wait, s_rdy, ld, turn, p]")
-            print(t[2 * w + a, lo:hi][:, [0, 1, 2, 6, 5]] - base)
+            print(f"softmax group {a} warp {w}: [wait, s_rdy, ld, p]")
+            print(t[2 * w + a, lo:hi][:, [0, 1, 2, 5]] - base)
     for a in (0, 1):
         print(f"MMA issuer {a}: [wait_p, got_p, -, got_turn, pv, qk]")
         print(t[8 + a, lo:hi, :6] - base)
