@@ -284,11 +284,9 @@ __device__ __forceinline__ void exp2_poly_pair(uint64_t x2, float& p0, float& p1
 
 // --------------------------------------------------------------------------------------
 // Softmax of one 128 x 128 score tile with one thread per query row (a warpgroup per query
-// tile); no data crosses threads.  The running maximum is only raised when it grows by more
-// than 2^kRescaleThreshold, so the output accumulator is rescaled rarely; P stays below 2^8 in
-// between.  The caller has seen S of this tile complete, which (the tensor pipe runs in issue
-// order) also means the previous P V into O has landed, so O may be rescaled here without
-// another wait.
+// tile); no data crosses threads.  The caller has seen S of this tile complete, which (the
+// tensor pipe runs in issue order) also means the previous P V into O has landed, so O may be
+// rescaled here without another wait.
 // --------------------------------------------------------------------------------------
 __device__ __forceinline__ void group_barrier(int a) {
   if (a == 0) asm volatile("bar.sync 1, 128;" ::: "memory");
@@ -456,7 +454,7 @@ window_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
   const uint32_t bar_s_full = sBar + 32 + 16 * kStages;      // [2]  MMA warp a -> softmax a
   const uint32_t bar_p_full = bar_s_full + 16;               // [2]  softmax a -> MMA warp a (128 arrivals)
   const uint32_t bar_o_final = bar_p_full + 16;              // [2]  MMA warp a -> softmax a
-  const uint32_t bar_mturn = bar_o_final + 16;                 // [2]  MMA warp 1-a -> MMA warp a: your turn on the tensor pipe
+  const uint32_t bar_mturn = bar_o_final + 16;               // [2]  MMA warp 1-a -> MMA warp a: your turn on the tensor pipe
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(gen + kSmemBar + 224);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(gen + kSmemBar + 228);
   volatile int* merge_flag = reinterpret_cast<volatile int*>(gen + kSmemBar + 232);   // [2]
