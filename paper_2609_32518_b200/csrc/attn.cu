@@ -248,11 +248,14 @@ struct Waiter {
   }
 };
 
-// The CTA owns 384 x 168 registers; 128 x 96 + 256 x 200 stays inside that (an increase that
-// the pool cannot satisfy would wait forever).
-static_assert(128 * 96 + 256 * 200 <= 384 * 168, "register redistribution exceeds the CTA's allocation");
-__device__ __forceinline__ void reg_dealloc_96() { asm volatile("setmaxnreg.dec.sync.aligned.u32 96;"); }
-__device__ __forceinline__ void reg_alloc_200() { asm volatile("setmaxnreg.inc.sync.aligned.u32 200;"); }
+// The CTA owns 384 x 168 registers; 128 x 72 for the service warps + 256 x 216 for the softmax
+// warps uses exactly that (an increase that the pool cannot satisfy would wait forever).  216 is
+// what the softmax warps need to run without spills.
+constexpr int kRegsService = 72, kRegsSoftmax = 216;
+static_assert(128 * kRegsService + 256 * kRegsSoftmax <= 384 * 168, "register redistribution exceeds the CTA's allocation");
+static_assert(kRegsService == 72 && kRegsSoftmax == 216, "keep the setmaxnreg literals below in step");
+__device__ __forceinline__ void reg_dealloc_service() { asm volatile("setmaxnreg.dec.sync.aligned.u32 72;"); }
+__device__ __forceinline__ void reg_alloc_softmax() { asm volatile("setmaxnreg.inc.sync.aligned.u32 216;"); }
 
 // 2^x for a pair of floats without the MUFU pipe: x = n + f with n = round(x) (the add of
 // 1.5 * 2^23 leaves n in the low mantissa bits), 2^f by a cubic on [-0.5, 0.5] (relative error
@@ -491,7 +494,7 @@ window_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
   const Waiter w{abort_flag, kWaitCycles};
 
   if (warp >= 8) {
-    reg_dealloc_96();
+    reg_dealloc_service();
     if (warp == 10 && lane == 0) {
       // ------------------------------------------------------------ TMA producer
       prefetch_tensormap(&tm_q);
@@ -651,7 +654,7 @@ window_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
     // ---------------------------------------------------------------- softmax warpgroups
     // Warps 0-3 own query tile 0, warps 4-7 query tile 1; a thread owns a row from the scores
     // to the output.  The groups never wait for each other.
-    reg_alloc_200();
+    reg_alloc_softmax();
     const int a = warp >> 2;               // query tile of this warpgroup
     const int row = tid & 127;             // row inside the tile = TMEM lane
     const uint32_t t_lane = tmem_base + (static_cast<uint32_t>((warp & 3) * 32) << 16);
