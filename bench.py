@@ -370,7 +370,7 @@ def run_ours(args):
                      "peak_source": f"{peaks['source']} cuBLAS bf16 burst",
                      "frac_of_sustained": attn_tflops / peaks["bf16_tflops_sustained"],
                      "frac_of_nominal_2250": attn_tflops / 2250.0,
-                     "traffic": ATTN_DRAM_TRAFFIC_BYTES if (args.workload == WORKLOAD and args.window is None) else None},
+                     "traffic": ATTN_DRAM_TRAFFIC_BYTES if (args.workload == WORKLOAD and not args.window) else None},
         "append_roofline": {"kernel": "rmsnorm_rope_kv_append_kernel" if args.rmsnorm else "rope_kv_append_kernel", "bound": "hbm",
                             "achieved": append_bytes / (t_append * 1e-3) / 1e9, "peak": peaks["hbm_gbs"],
                             "unit": "GB/s", "frac": append_bytes / (t_append * 1e-3) / 1e9 / peaks["hbm_gbs"],
