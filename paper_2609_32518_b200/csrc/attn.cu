@@ -332,36 +332,43 @@ __device__ __forceinline__ void mask_block32(uint32_t* s, int col0, int nvalid) 
 }
 
 // Exponentials of the 128 scores of a row (TMEM columns t_S .. t_S + 127) against the reference
-// maximum m_run: keys 0..63 come in through `lo` (already in registers when lo_loaded), keys
-// 64..127 are fetched in two blocks of 32 while the first half is exponentiated.  Leaves P
-// (bf16 pairs) in p0 (keys 0..63) and p1 (keys 64..127) and returns the row's sum of P.
+// maximum: the scores come in blocks of 32 columns, each fetched while the block before it is
+// exponentiated (a block keeps the MUFU pipe busy for 256 clk, longer than a TMEM load takes), so
+// that only the first block's load is exposed.  Leaves P (bf16 pairs) in p0 (keys 0..63) and p1
+// (keys 64..127) and returns the row's sum of P.
 template <bool kMasked>
-__device__ __forceinline__ float exp_row(uint32_t t_S, const uint32_t* lo, float c, float neg_ms, int nvalid,
-                                         uint32_t* p0, uint32_t* p1) {
+__device__ __forceinline__ float exp_row(uint32_t t_S, float c, float neg_ms, int nvalid, uint32_t* p0,
+                                         uint32_t* p1) {
   const uint64_t c2 = pack_f32x2(c, c);
   const uint64_t nm2 = pack_f32x2(neg_ms, neg_ms);
   uint64_t acc[4] = {0ull, 0ull, 0ull, 0ull};
-  uint32_t h0[32], h1[32];
-  tmem_ld32(t_S + 64, h0);             // keys 64..95, in flight during the first half
-  exp_block32(lo, p0, c2, nm2, acc);
-  exp_block32(lo + 32, p0 + 16, c2, nm2, acc);
+  uint32_t a[32], b[32];
+  tmem_ld32(t_S, a);
   tc_wait_ld();
-  tmem_ld32(t_S + 96, h1);             // keys 96..127
-  mask_block32<kMasked>(h0, 64, nvalid);
-  exp_block32(h0, p1, c2, nm2, acc);
+  tmem_ld32(t_S + 32, b);
+  mask_block32<kMasked>(a, 0, nvalid);
+  exp_block32(a, p0, c2, nm2, acc);
   tc_wait_ld();
-  mask_block32<kMasked>(h1, 96, nvalid);
-  exp_block32(h1, p1 + 16, c2, nm2, acc);
+  tmem_ld32(t_S + 64, a);
+  mask_block32<kMasked>(b, 32, nvalid);
+  exp_block32(b, p0 + 16, c2, nm2, acc);
+  tc_wait_ld();
+  tmem_ld32(t_S + 96, b);
+  mask_block32<kMasked>(a, 64, nvalid);
+  exp_block32(a, p1, c2, nm2, acc);
+  tc_wait_ld();
+  mask_block32<kMasked>(b, 96, nvalid);
+  exp_block32(b, p1 + 16, c2, nm2, acc);
   const uint64_t t = add_f32x2(add_f32x2(acc[0], acc[1]), add_f32x2(acc[2], acc[3]));
   float t0, t1;
   unpack_f32x2(t, t0, t1);
   return t0 + t1;
 }
 
-// Row maximum of the 128 scores in TMEM; leaves keys 0..63 (masked) in `lo`.
+// Row maximum of the 128 scores in TMEM.
 template <bool kMasked>
-__device__ __forceinline__ float max_row(uint32_t t_S, uint32_t* lo, int nvalid) {
-  uint32_t hi[64];
+__device__ __forceinline__ float max_row(uint32_t t_S, int nvalid) {
+  uint32_t hi[64], lo[64];
   tmem_ld32(t_S + 64, hi);
   tmem_ld32(t_S + 96, hi + 32);
   tmem_ld32(t_S, lo);
@@ -391,23 +398,13 @@ template <bool kMasked>
 __device__ __forceinline__ void softmax_row_tile(uint32_t t_S, uint32_t t_O, float c, int nvalid,
                                                  bool first, float& m_run, float& l_run,
                                                  uint32_t bar_p_full, int trace_role, int trace_tile) {
-  uint32_t lo[64];
-  if (first) {
-    m_run = max_row<kMasked>(t_S, lo, nvalid);
-  } else {
-    tmem_ld32(t_S, lo);
-    tmem_ld32(t_S + 32, lo + 32);
-    tc_wait_ld();
-    mask_block32<kMasked>(lo, 0, nvalid);
-    mask_block32<kMasked>(lo + 32, 32, nvalid);
-  }
+  if (first) m_run = max_row<kMasked>(t_S, nvalid);
   TRACE(trace_role, trace_tile, 2);
-  const float neg_ms = -m_run * c;
   uint32_t p0[32], p1[32];
-  float sum = exp_row<kMasked>(t_S, lo, c, neg_ms, nvalid, p0, p1);
+  float sum = exp_row<kMasked>(t_S, c, -m_run * c, nvalid, p0, p1);
   const bool redo = !first && !(sum <= kOptimisticLimit);   // also taken for inf and NaN
   if (__any_sync(0xFFFFFFFFu, redo)) {
-    const float mx = max_row<kMasked>(t_S, lo, nvalid);
+    const float mx = max_row<kMasked>(t_S, nvalid);
     float alpha = 1.f;
     if (mx > m_run) {
       alpha = ex2((m_run - mx) * c);
@@ -423,7 +420,7 @@ __device__ __forceinline__ void softmax_row_tile(uint32_t t_S, uint32_t t_O, flo
       for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
       tmem_st32(t_O + q * 32, o);
     }
-    sum = exp_row<kMasked>(t_S, lo, c, -m_run * c, nvalid, p0, p1);
+    sum = exp_row<kMasked>(t_S, c, -m_run * c, nvalid, p0, p1);
   }
   tmem_st32(t_S, p0);        // P of keys 0..63 over score columns 0..31
   tmem_st32(t_S + 32, p1);   // P of keys 64..127 over score columns 32..63
