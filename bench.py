@@ -35,7 +35,7 @@ METRIC = "windowed-attn TFLOP/s at 1.3B-class shape (whole layer-chunk step: tab
 WORKLOAD = "cfg2"
 # dram__bytes_read.sum + dram__bytes_write.sum of one window_attn launch at this workload,
 # from the ncu capture summarised under profiles/ (None until captured)
-ATTN_DRAM_TRAFFIC_BYTES = 391_794_688
+ATTN_DRAM_TRAFFIC_BYTES = 286_214_400
 
 
 def load_peaks():
