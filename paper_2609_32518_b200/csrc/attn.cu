@@ -344,19 +344,19 @@ __device__ __forceinline__ float exp_row(uint32_t t_S, float c, float neg_ms, in
   uint64_t acc[4] = {0ull, 0ull, 0ull, 0ull};
   uint32_t a[32], b[32];
   tmem_ld32(t_S, a);
-  tc_wait_ld();
+  tc_wait_ld32(a);
   tmem_ld32(t_S + 32, b);
   mask_block32<kMasked>(a, 0, nvalid);
   exp_block32(a, p0, c2, nm2, acc);
-  tc_wait_ld();
+  tc_wait_ld32(b);
   tmem_ld32(t_S + 64, a);
   mask_block32<kMasked>(b, 32, nvalid);
   exp_block32(b, p0 + 16, c2, nm2, acc);
-  tc_wait_ld();
+  tc_wait_ld32(a);
   tmem_ld32(t_S + 96, b);
   mask_block32<kMasked>(a, 64, nvalid);
   exp_block32(a, p1, c2, nm2, acc);
-  tc_wait_ld();
+  tc_wait_ld32(b);
   mask_block32<kMasked>(b, 96, nvalid);
   exp_block32(b, p1 + 16, c2, nm2, acc);
   const uint64_t t = add_f32x2(add_f32x2(acc[0], acc[1]), add_f32x2(acc[2], acc[3]));
@@ -373,7 +373,10 @@ __device__ __forceinline__ float max_row(uint32_t t_S, int nvalid) {
   tmem_ld32(t_S + 96, hi + 32);
   tmem_ld32(t_S, lo);
   tmem_ld32(t_S + 32, lo + 32);
-  tc_wait_ld();
+  tc_wait_ld32(hi);
+  reg_fence32(hi + 32);
+  reg_fence32(lo);
+  reg_fence32(lo + 32);
   mask_block32<kMasked>(hi, 64, nvalid);
   mask_block32<kMasked>(hi + 32, 96, nvalid);
   mask_block32<kMasked>(lo, 0, nvalid);
@@ -415,7 +418,7 @@ __device__ __forceinline__ void softmax_row_tile(uint32_t t_S, uint32_t t_O, flo
     for (int q = 0; q < 4; ++q) {
       uint32_t o[32];
       tmem_ld32(t_O + q * 32, o);
-      tc_wait_ld();
+      tc_wait_ld32(o);
 #pragma unroll
       for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
       tmem_st32(t_O + q * 32, o);
@@ -714,7 +717,7 @@ window_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
           for (int q = 0; q < 4; ++q) {
             float o[32];
             tmem_ld32(t_O + q * 32, reinterpret_cast<uint32_t*>(o));
-            tc_wait_ld();
+            tc_wait_ld32(reinterpret_cast<uint32_t*>(o));
             if (n < p.L) store_row(dst + 4 * q, o, inv_l);
           }
         }
@@ -744,7 +747,7 @@ window_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
           for (int q = 0; q < 4; ++q) {
             uint32_t o[32];
             tmem_ld32(t_O + q * 32, o);
-            tc_wait_ld();
+            tc_wait_ld32(o);
 #pragma unroll
             for (int i = 0; i < 32; ++i) mine[(q * 32 + i) * 128 + row] = __uint_as_float(o[i]);
           }
@@ -786,7 +789,7 @@ window_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
               float m_c;
               if (c == me) {
                 tmem_ld32(t_O + 32 * q, reinterpret_cast<uint32_t*>(v));
-                tc_wait_ld();
+                tc_wait_ld32(reinterpret_cast<uint32_t*>(v));
                 m_c = m_run;
               } else {
                 const float* pc = part_of(c);
