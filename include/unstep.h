@@ -81,8 +81,8 @@ int unstep_rope_table(const unstep_shape_t* shape, int32_t start_frame, float* c
  * same entries).
  *
  * For every stream b, token n, head h, pair j, with c = cos[n][j], s = sin[n][j]:
- *     y_even = fl32(fl32(x_even*c) - fl32(x_odd*s))
- *     y_odd  = fl32(fl32(x_even*s) + fl32(x_odd*c))        (no fused multiply-add)
+ *     y[2j]   = fl32(fl32(x[2j]*c) - fl32(x[2j+1]*s))
+ *     y[2j+1] = fl32(fl32(x[2j]*s) + fl32(x[2j+1]*c))      (no fused multiply-add)
  * rounded to bf16 (nearest even).  q_out = rot(q_in); ring_k[b][slot][t] = rot(k_in),
  * ring_v[b][slot][t] = v_in (bit copy), slot = (start_frame[b] + f) mod C, where
  * n = f*T + t.  Slots of other frames are not touched.
@@ -119,7 +119,13 @@ int unstep_rope_kv_append(const unstep_shape_t* shape, const int32_t* start_fram
  * Scratch: work items that are split across thread blocks exchange partial results through a
  * buffer the library keeps per (device, stream).  The first call on a stream creates it with
  * cudaMalloc (about 40 MB): make that call outside any stream capture.  Calls on one stream
- * share the buffer safely; calls on different streams use different buffers.
+ * share the buffer safely; calls on different streams use different buffers.  A buffer is replaced
+ * by a larger one when a later call on its stream needs more (more SMs or more work items).
+ * CUDA graphs: a call captured into a graph freezes the addresses of the capture stream's buffer
+ * into the graph.  Such a graph is invalid after unstep_shutdown() and after a larger problem was
+ * run on the capture stream (both free the buffer), and its replays must not overlap on the GPU
+ * with each other or with direct calls on the capture stream.  Capture all graphs that may replay
+ * back to back on one stream, after one uncaptured call of the largest problem on that stream.
  */
 int unstep_window_attn(const unstep_shape_t* shape, const int32_t* start_frame,
                        int32_t window_frames, const void* q_rot, const void* ring_k,
@@ -155,9 +161,8 @@ int unstep_window_attn_sink(const unstep_shape_t* shape, int32_t sink_frames,
 
 /*
  * RMS normalisation of q and k fused in front of the rotation (appendix "Diffusion transformer
- * runtime": queries and keys are split into heads "after linear projection and RMS
- * normalization"; the paper gives no formula, this is the textbook RMSNorm over the whole token
- * vector of Hn*128 channels with a learned gain):
+ * runtime": q and k are normalised before they are split into heads; the paper gives no formula,
+ * this is the textbook RMSNorm over the whole token vector of Hn*128 channels with a learned gain):
  *     y = x / sqrt(mean(x^2) + eps) * gain,   rounded to bf16, then rotated and appended exactly
  * as unstep_rope_kv_append_sink does (v is copied, not normalised).  The mean of squares is
  * accumulated in double and rounded to float32; sqrt, reciprocal and the two products are single
@@ -203,6 +208,31 @@ int unstep_window_attn_noalloc(const unstep_shape_t* shape, const int32_t* start
                                int32_t window_frames, const void* q_rot, const void* ring_k,
                                const void* ring_v, void* out, void* cuda_stream);
 
+/*
+ * The work split of one unstep_window_attn(_sink) launch, listed on the host by the same integer
+ * code that the kernel's roles run on the device (the paper has no counterpart: a diagnostic for
+ * tests and tuning).  No device is touched and no GPU is needed.
+ *
+ * The launch is cut into work items (stream, head, pair of 128-query tiles); an item has one step
+ * per 128-key tile of its window.  Each of at most `max_workers` workers (one per SM) first takes
+ * whole items round-robin; what is left over is one sequence of steps cut into equal contiguous
+ * shares, so an item there may be split along its keys into parts that different workers compute
+ * and the last one to finish merges.
+ *
+ *   segs     : HOST int32 [max_segs][10], written (may be NULL when max_segs is 0).  One row per
+ *              segment in the order the worker walks them: worker, stream, head, query pair,
+ *              query tiles in the pair (1 or 2), first key tile, end key tile (exclusive), key
+ *              tiles of the whole item, number of parts the item is split into (1 = whole), and the
+ *              scratch slot (0 or 1) the part is published in (-1 for a whole item).
+ *   n_segs   : HOST int32, written: the number of segments of the launch (may exceed max_segs; only
+ *              the first max_segs rows are written).
+ * Only the first launch of the call is listed (the first 32 streams).  Arguments are checked as in
+ * unstep_window_attn_sink; sink_frames = 0 lists the plain rolling window.
+ */
+int unstep_window_attn_plan(const unstep_shape_t* shape, int32_t sink_frames, const int32_t* start_frame,
+                            int32_t recent_frames, int32_t sink_attend, int32_t max_workers,
+                            int32_t* segs, int32_t max_segs, int32_t* n_segs);
+
 /* Static, human-readable text for a status code. */
 const char* unstep_strerror(int code);
 
@@ -230,6 +260,17 @@ void unstep_shutdown(void);
 
 /* Number of kernels the library has launched in this process (all devices). */
 int64_t unstep_launch_count(void);
+
+#ifdef UNSTEP_TRACE
+/*
+ * Only in a library built with -DUNSTEP_TRACE (a diagnostic build, slower): the attention kernel
+ * stamps the clock at the hand-overs between its roles.  Both calls synchronise the device and
+ * copy the stamps of the last launch to HOST memory: [12 roles][64 key tiles][8 events] clock64
+ * values of thread block 0, and [160 thread blocks][16 events] global-timer values.
+ */
+int unstep_debug_read_trace(long long* host_out);
+int unstep_debug_read_cta_trace(unsigned long long* host_out);
+#endif
 
 #ifdef __cplusplus
 }

@@ -406,9 +406,9 @@ def explicit_frames_attn(history: ExplicitHistory, frames, q_rot_bits: np.ndarra
 
 # ---------------------------------------------------------------------------
 # RMS normalisation of q and k in front of the rotation (appendix "Diffusion transformer
-# runtime": queries and keys are reshaped into heads "after linear projection and RMS
-# normalization").  The paper gives no formula; this is the textbook RMSNorm over the whole
-# token vector (all heads, Hn*128 wide) with a learned per-channel gain:
+# runtime": q and k pass through the projection and an RMS norm before the head split).  The
+# paper gives no formula; this is the textbook RMSNorm over the whole token vector (all heads,
+# Hn*128 wide) with a learned per-channel gain:
 #     y = x / sqrt(mean(x^2) + eps) * g
 # Readings: the mean of squares is accumulated in float64 (so that it does not depend on the
 # order of summation) and rounded to float32; sqrt, reciprocal and the two products are single

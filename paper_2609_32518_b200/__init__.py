@@ -15,6 +15,7 @@ from .binding import (  # noqa: F401
     rope_kv_append_sink,
     window_attn_sink,
     rmsnorm_rope_kv_append,
+    window_attn_plan,
     poll_status,
     shutdown,
     selftest_wait_limit,

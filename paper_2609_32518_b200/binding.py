@@ -9,7 +9,7 @@ from . import build as _build
 
 EXPORTS = ("unstep_rope_table", "unstep_rope_kv_append", "unstep_window_attn",
            "unstep_window_attn_noalloc", "unstep_rope_kv_append_sink", "unstep_window_attn_sink",
-           "unstep_rmsnorm_rope_kv_append", "unstep_selftest_wait_limit", "unstep_shutdown", "unstep_strerror", "unstep_poll_status", "unstep_launch_count")
+           "unstep_rmsnorm_rope_kv_append", "unstep_window_attn_plan", "unstep_selftest_wait_limit", "unstep_shutdown", "unstep_strerror", "unstep_poll_status", "unstep_launch_count")
 
 
 class UnstepError(RuntimeError):
@@ -72,6 +72,9 @@ def lib() -> ctypes.CDLL:
                                                     c_void_p, c_void_p, c_void_p, c_void_p, c_float,
                                                     c_void_p, c_void_p, c_int64, c_void_p, c_void_p,
                                                     c_void_p, c_void_p]
+        L.unstep_window_attn_plan.restype = c_int
+        L.unstep_window_attn_plan.argtypes = [POINTER(Shape), c_int32, POINTER(c_int32), c_int32, c_int32,
+                                              c_int32, POINTER(c_int32), c_int32, POINTER(c_int32)]
         L.unstep_selftest_wait_limit.restype = c_int
         L.unstep_selftest_wait_limit.argtypes = [c_int64, c_void_p]
         L.unstep_shutdown.restype = None
@@ -228,6 +231,21 @@ def window_attn_sink(shape: Shape, sink_frames: int, start_frame, recent_frames:
         int(sink_attend), _dev_ptr(q_rot, bf, n, "q_rot"), _dev_ptr(cache_k, bf, nr, "cache_k"),
         _dev_ptr(cache_v, bf, nr, "cache_v"), _dev_ptr(out, bf, n, "out"), _stream_ptr(stream)),
         "unstep_window_attn_sink")
+
+
+def window_attn_plan(shape: Shape, start_frame, recent_frames: int, max_workers: int, sink_frames: int = 0,
+                     sink_attend: int = 0):
+    """unstep_window_attn_plan: the segments of one attention launch as rows of 10 ints (worker,
+    stream, head, query pair, query tiles, first key tile, end key tile, tiles of the item, parts,
+    scratch slot).  Host only."""
+    n = c_int32(0)
+    starts = _starts(shape, start_frame)
+    args = (ctypes.byref(shape), int(sink_frames), starts, int(recent_frames), int(sink_attend),
+            int(max_workers))
+    _check(lib().unstep_window_attn_plan(*args, None, 0, ctypes.byref(n)), "unstep_window_attn_plan")
+    buf = (c_int32 * (10 * max(n.value, 1)))()
+    _check(lib().unstep_window_attn_plan(*args, buf, n.value, ctypes.byref(n)), "unstep_window_attn_plan")
+    return [tuple(buf[10 * i:10 * i + 10]) for i in range(n.value)]
 
 
 def selftest_wait_limit(limit_cycles: int, stream=None):

@@ -27,6 +27,7 @@
 
 #include "common.h"
 #include "ptx.cuh"
+#include "attn_sched.h"
 
 namespace unstep {
 
@@ -64,8 +65,6 @@ __device__ __forceinline__ unsigned long long gtime() {
   } while (0)
 #endif
 
-constexpr int kTileM = 128;                 // queries per tile (two tiles per work item)
-constexpr int kTileN = 128;                 // keys per tile
 constexpr int kHalfBytes = 128 * 64 * 2;    // one TMA box: 128 rows x 64 bf16 (128-byte rows)
 constexpr int kTileBytes = 2 * kHalfBytes;  // 128 x 128 bf16
 constexpr int kStages = 5;                  // 32 KB buffers shared by the K and V tiles
@@ -78,154 +77,10 @@ constexpr int kSmemKV = 2 * kTileBytes;
 constexpr int kSmemBar = kSmemKV + kStages * kTileBytes;
 constexpr int kAttnSmemBytes = kSmemBar + 256;
 
-struct AttnParams {
-  int32_t Hn, L, T, C;
-  int32_t q_tiles;          // ceil(L / 128)
-  int32_t q_pairs;          // ceil(q_tiles / 2)
-  int32_t tiles_per_frame;  // ceil(T / 128)
-  int32_t flat;             // 1: key tiles run across frame boundaries inside a slot run
-  int32_t n_streams;
-  float scale_log2e;        // log2(e) / sqrt(128)
-  int32_t items_per_stream; // Hn * q_pairs
-  int32_t full_rounds;      // whole rounds per stream: items_per_stream / gridDim.x
-  int64_t total_steps;      // remainder: sum over the leftover items of their key tiles
-  float* part;              // workspace: partial results of split items, kPartFloats per slot
-  int* counters;            // workspace: arrivals per (item, query tile), zero between launches
-  int32_t sink;             // S: cache slots [0, S) hold frames [0, S) for good, the ring follows
-  int32_t first_frame[kMaxStreamsPerLaunch];  // first frame of the recent part of stream b
-  int32_t n_sink[kMaxStreamsPerLaunch];       // sink frames attended in front of the recent part
-  int32_t tiles[kMaxStreamsPerLaunch];        // key tiles of one item of stream b
-  // flat mode: the attended frames are at most three runs of consecutive cache slots (sink
-  // prefix, ring up to its end, ring from its start); run r starts at cache row run_row0 and
-  // has run_rows keys, its tiles are [run_tile_end[r-1], run_tile_end[r])
-  int32_t run_row0[kMaxStreamsPerLaunch][3];
-  int32_t run_rows[kMaxStreamsPerLaunch][3];
-  int32_t run_tile_end[kMaxStreamsPerLaunch][3];
-  int64_t step_base[kMaxStreamsPerLaunch];    // remainder steps of all streams before b
-};
-
 // Partial result of one query tile of a split item: O[col][row] (unnormalised, relative to the
 // part's own reference maximum), then m[row], l[row].  Two tiles per slot, two slots per CTA.
 constexpr int kPartTileFloats = 128 * 128 + 2 * 128;
 constexpr int kPartFloats = 2 * kPartTileFloats;
-constexpr int kMinStepsPerCta = 4;
-
-// One unit of work of a CTA: key tiles [t0, t1) of item (b, h, query-tile pair qp).
-struct Seg {
-  int b, h, qp, nq, t0, t1;
-  int tiles;          // key tiles of the whole item
-  int item;           // item index inside the launch
-  int64_t item_step0; // global step index of the item's first tile
-  bool first_in_cta;  // this segment starts the CTA's range
-};
-
-// Where key tile j of an item of stream b lives and how many of its 128 keys are real.
-// Flat mode: tiles are cut from the runs of consecutive ring slots, so only the last tile of
-// a run is ragged; it is fetched through the per-frame map, whose zero fill ends it cleanly at
-// the end of its frame (a run ends on a frame end, and the ragged tile is shorter than a frame).
-// Per-frame mode (frames shorter than a tile): every tile lies inside one frame.
-struct TileInfo {
-  int valid;      // real keys in the tile, 1..128
-  bool framed;    // fetch through the (token, slot) map at (tok0, slot), else the flat map at row
-  int row, slot, tok0;
-};
-__device__ __forceinline__ TileInfo tile_info(const AttnParams& p, int b, int j) {
-  TileInfo t;
-  if (p.flat) {
-    int r = 0;
-    if (j >= p.run_tile_end[b][0]) r = (j >= p.run_tile_end[b][1]) ? 2 : 1;
-    const int t_begin = r == 0 ? 0 : p.run_tile_end[b][r - 1];
-    const int tt = j - t_begin;
-    const int rows = p.run_rows[b][r];
-    const int row0 = p.run_row0[b][r];
-    const int ntl = p.run_tile_end[b][r] - t_begin;
-    const bool last = (tt == ntl - 1);
-    t.valid = last ? rows - kTileN * tt : kTileN;
-    t.framed = last;
-    t.row = row0 + kTileN * tt;
-    t.slot = (row0 + rows - 1) / p.T;
-    t.tok0 = p.T - t.valid;
-  } else {
-    const int fi = j / p.tiles_per_frame;
-    const int tt = j - fi * p.tiles_per_frame;
-    t.valid = (tt == p.tiles_per_frame - 1) ? p.T - kTileN * tt : kTileN;
-    t.framed = true;
-    t.row = 0;
-    // frame list = the attended sink frames, then the recent frames
-    const int frame = fi < p.n_sink[b] ? fi : p.first_frame[b] + fi - p.n_sink[b];
-    t.slot = frame < p.sink ? frame : p.sink + (frame - p.sink) % p.C;
-    t.tok0 = kTileN * tt;
-  }
-  return t;
-}
-
-// Work split.  Items are ordered stream, head, query pair, so neighbouring CTAs work on the
-// same head and share its K/V through L2.
-//   1. Whole rounds: while a stream still has at least gridDim.x items, CTA c takes item
-//      (round * gridDim.x + c) whole.  All CTAs walk the key tiles in step, so a K/V tile is
-//      fetched from HBM once and then hit in L2 by the other CTAs of the head.
-//   2. Remainder: the leftover items of all streams (fewer than gridDim.x per stream) form one
-//      sequence of (item, key tile) steps, and every CTA takes an equal contiguous share of
-//      it.  An item that straddles a CTA boundary is split along its keys; the parts are
-//      merged by whichever CTA finishes last.  Only a few heads are live here, so their K/V
-//      stays in L2 although the CTAs are no longer in step.
-struct Sched {
-  int64_t lo, hi, cur;
-  int b_round, round;   // position in the whole rounds
-  const AttnParams& p;
-  __device__ static int64_t cta_lo(const AttnParams& p, int64_t c) { return p.total_steps * c / gridDim.x; }
-  __device__ static int cta_of(const AttnParams& p, int64_t step) {
-    int64_t c = step * gridDim.x / p.total_steps;
-    while (c + 1 < gridDim.x && cta_lo(p, c + 1) <= step) ++c;
-    while (c > 0 && cta_lo(p, c) > step) --c;
-    return static_cast<int>(c);
-  }
-  __device__ Sched(const AttnParams& prm) : p(prm) {
-    lo = cta_lo(p, blockIdx.x);
-    hi = cta_lo(p, blockIdx.x + 1);
-    cur = lo;
-    b_round = 0;
-    round = 0;
-  }
-  __device__ void decode(Seg& s, int b, int in_stream) const {
-    s.b = b;
-    s.tiles = p.tiles[b];
-    s.item = b * p.items_per_stream + in_stream;
-    s.qp = in_stream % p.q_pairs;
-    s.h = in_stream / p.q_pairs;
-    s.nq = (2 * s.qp + 1 < p.q_tiles) ? 2 : 1;
-  }
-  __device__ bool next(Seg& s) {
-    while (b_round < p.n_streams) {          // whole rounds
-      if (round < p.full_rounds) {
-        decode(s, b_round, round * static_cast<int>(gridDim.x) + static_cast<int>(blockIdx.x));
-        s.t0 = 0;
-        s.t1 = s.tiles;
-        s.item_step0 = 0;
-        s.first_in_cta = false;
-        ++round;
-        return true;
-      }
-      round = 0;
-      ++b_round;
-    }
-    if (cur >= hi) return false;             // remainder
-    int b = 0;
-    while (b + 1 < p.n_streams && p.step_base[b + 1] <= cur) ++b;
-    const int tiles = p.tiles[b];
-    const int64_t rel = cur - p.step_base[b];
-    const int left_item = static_cast<int>(rel / tiles);
-    decode(s, b, p.full_rounds * static_cast<int>(gridDim.x) + left_item);
-    s.t0 = static_cast<int>(rel - static_cast<int64_t>(left_item) * tiles);
-    const int64_t left = hi - cur;
-    s.t1 = (left < tiles - s.t0) ? s.t0 + static_cast<int>(left) : tiles;
-    s.item_step0 = cur - s.t0;
-    s.first_in_cta = (cur == lo);
-    cur += s.t1 - s.t0;
-    return true;
-  }
-};
-
 struct Waiter {
   volatile int* abort_flag;
   long long limit;   // clock cycles after which a wait gives up
@@ -257,34 +112,6 @@ static_assert(kRegsService == 72 && kRegsSoftmax == 216, "keep the setmaxnreg li
 __device__ __forceinline__ void reg_dealloc_service() { asm volatile("setmaxnreg.dec.sync.aligned.u32 72;"); }
 __device__ __forceinline__ void reg_alloc_softmax() { asm volatile("setmaxnreg.inc.sync.aligned.u32 216;"); }
 
-// 2^x for a pair of floats without the MUFU pipe: x = n + f with n = round(x) (the add of
-// 1.5 * 2^23 leaves n in the low mantissa bits), 2^f by a cubic on [-0.5, 0.5] (relative error
-// 7.5e-5, far below the bf16 rounding of P), and n is added into the exponent field.
-// Inputs are clamped to [-126, 127] so that the exponent never wraps: -inf gives about 1e-38,
-// anything above 127 gives 2^127, which the caller's check of the row sum then catches.
-__device__ __forceinline__ void exp2_poly_pair(uint64_t x2, float& p0, float& p1) {
-  float x0, x1;
-  unpack_f32x2(x2, x0, x1);
-  const uint64_t xc = pack_f32x2(fminf(fmaxf(x0, -126.f), 127.f), fminf(fmaxf(x1, -126.f), 127.f));
-  const uint64_t magic = pack_f32x2(12582912.f, 12582912.f);
-  const uint64_t t2 = add_f32x2(xc, magic);
-  const uint64_t n2 = add_f32x2(t2, pack_f32x2(-12582912.f, -12582912.f));
-  const uint64_t f2 = fma_f32x2(n2, pack_f32x2(-1.f, -1.f), xc);
-  uint64_t q2 = fma_f32x2(f2, pack_f32x2(0.055171650f, 0.055171650f), pack_f32x2(0.24261113f, 0.24261113f));
-  q2 = fma_f32x2(q2, f2, pack_f32x2(0.69326097f, 0.69326097f));
-  q2 = fma_f32x2(q2, f2, pack_f32x2(0.99992806f, 0.99992806f));
-  float q0, q1, t0, t1;
-  unpack_f32x2(q2, q0, q1);
-  unpack_f32x2(t2, t0, t1);
-  p0 = __uint_as_float(__float_as_uint(q0) + (__float_as_uint(t0) << 23));
-  p1 = __uint_as_float(__float_as_uint(q1) + (__float_as_uint(t1) << 23));
-}
-
-#ifndef UNSTEP_EMU_OF8
-#define UNSTEP_EMU_OF8 0   // of every 8 column pairs, this many take the polynomial instead of MUFU
-#endif
-
-
 // --------------------------------------------------------------------------------------
 // Softmax of one 128 x 128 score tile with one thread per query row (a warpgroup per query
 // tile); no data crosses threads.  The caller has seen S of this tile complete, which (the
@@ -302,16 +129,9 @@ __device__ __forceinline__ void exp_block32(const uint32_t* s, uint32_t* p, uint
 #pragma unroll
   for (int i = 0; i < 16; ++i) {
     const uint64_t x2 = fma_f32x2(pack_f32x2(__uint_as_float(s[2 * i]), __uint_as_float(s[2 * i + 1])), c2, nm2);
-    float p0, p1;
-    if ((i & 7) < UNSTEP_EMU_OF8) {
-      // part of the exponentials runs on the FMA pipe: the MUFU pipe alone would bound the tile
-      exp2_poly_pair(x2, p0, p1);
-    } else {
-      float x0, x1;
-      unpack_f32x2(x2, x0, x1);
-      p0 = ex2(x0);
-      p1 = ex2(x1);
-    }
+    float x0, x1;
+    unpack_f32x2(x2, x0, x1);
+    const float p0 = ex2(x0), p1 = ex2(x1);
     acc[i & 3] = add_f32x2(acc[i & 3], pack_f32x2(p0, p1));
     p[i] = pack_bf16x2(p0, p1);
   }
@@ -502,7 +322,7 @@ window_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
       prefetch_tensormap(&tm_v);
       prefetch_tensormap(&tm_kf);
       prefetch_tensormap(&tm_vf);
-      Sched sched(p);
+      Sched sched(p, static_cast<int>(blockIdx.x));
       Seg s;
       uint32_t kv_it = 0, q_it[2] = {0, 0};
       bool ok = true;
@@ -544,7 +364,7 @@ window_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
       // tile: O_a += P_a V (two halves, as P arrives), then S_a = Q_a K_next^T.  Both warps
       // walk the same K/V ring; a stage is released when both have retired it.
       const int a = warp - 8;
-      Sched sched(p);
+      Sched sched(p, static_cast<int>(blockIdx.x));
       Seg s;
       uint32_t kv_it = 0, q_it = 0, sp_it = 0, mturn_it = 0;
       bool ok = true;
@@ -661,7 +481,7 @@ window_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
     const uint32_t t_S = t_lane + a * 128, t_O = t_lane + 256 + a * 128;
     const uint32_t my_p_full = bar_p_full + 8 * a;
     volatile int* my_flag = merge_flag + a;
-    Sched sched(p);
+    Sched sched(p, static_cast<int>(blockIdx.x));
     Seg s;
     uint32_t it = 0, seg_it = 0;
     bool ok = true;
@@ -728,8 +548,8 @@ window_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         // A part that finds all others already published merges at once without publishing
         // itself; otherwise it publishes (O, m, l), counts itself in, and merges if that made
         // the count complete.
-        const int c_lo = Sched::cta_of(p, s.item_step0);
-        const int c_hi = Sched::cta_of(p, s.item_step0 + s.tiles - 1);
+        const int c_lo = first_part_worker(p, s);
+        const int c_hi = last_part_worker(p, s);
         const int others = c_hi - c_lo;
         int* counter = p.counters + 2 * s.item + a;
         if (row == 0 && ok) {
@@ -741,7 +561,7 @@ window_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         if (*abort_flag) break;            // raised before the barrier by whoever gave up
         bool last = (*my_flag != 0);
         if (!last) {
-          float* mine = p.part + (static_cast<int64_t>(2 * blockIdx.x + (s.first_in_cta ? 0 : 1)) * kPartFloats +
+          float* mine = p.part + (static_cast<int64_t>(2 * blockIdx.x + (s.first_in_worker ? 0 : 1)) * kPartFloats +
                                   a * kPartTileFloats);
 #pragma unroll
           for (int q = 0; q < 4; ++q) {
@@ -755,18 +575,24 @@ window_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
           mine[128 * 128 + 128 + row] = l_run;
           __threadfence();
           group_barrier(a);   // all of this part is published; everyone has read the flag
-          if (row == 0) *my_flag = (atomicAdd(counter, 1) == others) ? 1 : 0;
+          if (row == 0) {
+            // release: the group's stores (fenced above, ordered before this thread by the barrier)
+            // become visible before the count; acquire: a merging part sees the other parts' stores
+            __threadfence();
+            const int before = atomicAdd(counter, 1);
+            __threadfence();
+            *my_flag = (before == others) ? 1 : 0;
+          }
           group_barrier(a);
           last = (*my_flag != 0);
         }
         if (last) {
-          __threadfence();
+          __threadfence();   // acquire side for every thread that reads the other parts below
           if (row == 0) *counter = 0;   // ready for the next launch
           const int me = static_cast<int>(blockIdx.x);
           auto part_of = [&](int c) -> const float* {
-            const int64_t clo = Sched::cta_lo(p, c);
-            const bool first = clo >= s.item_step0;   // the part starts the range of CTA c
-            return p.part + (static_cast<int64_t>(2 * c + (first ? 0 : 1)) * kPartFloats + a * kPartTileFloats);
+            return p.part + (static_cast<int64_t>(2 * c + part_slot(p, c, s.item_step0)) * kPartFloats +
+                             a * kPartTileFloats);
           };
           float m_all = m_run;
           for (int c = c_lo; c <= c_hi; ++c)
@@ -915,28 +741,30 @@ struct Workspace {
 static std::mutex g_ws_mutex;
 static std::map<std::pair<int, cudaStream_t>, Workspace> g_workspaces;
 
-static bool get_workspace(cudaStream_t st, size_t slots, size_t n_counters, Workspace* out) {
+static int get_workspace(cudaStream_t st, size_t slots, size_t n_counters, Workspace* out) {
   int dev = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess) return false;
+  if (cudaGetDevice(&dev) != cudaSuccess) return UNSTEP_ERR_CUDA;
   std::lock_guard<std::mutex> lock(g_ws_mutex);
   Workspace& ws = g_workspaces[std::make_pair(dev, st)];
   if (ws.slots < slots) {
-    if (ws.part != nullptr && cudaFree(ws.part) != cudaSuccess) return false;
+    if (ws.part != nullptr && cudaFree(ws.part) != cudaSuccess) return UNSTEP_ERR_CUDA;
     ws.part = nullptr;
     ws.slots = 0;
-    if (cudaMalloc(&ws.part, slots * kPartFloats * sizeof(float)) != cudaSuccess) return false;
+    if (cudaMalloc(&ws.part, slots * kPartFloats * sizeof(float)) != cudaSuccess) return UNSTEP_ERR_CUDA;
     ws.slots = slots;
   }
   if (ws.n_counters < n_counters) {
-    if (ws.counters != nullptr && cudaFree(ws.counters) != cudaSuccess) return false;
+    if (ws.counters != nullptr && cudaFree(ws.counters) != cudaSuccess) return UNSTEP_ERR_CUDA;
     ws.counters = nullptr;
     ws.n_counters = 0;
-    if (cudaMalloc(&ws.counters, n_counters * sizeof(int)) != cudaSuccess) return false;
-    if (cudaMemset(ws.counters, 0, n_counters * sizeof(int)) != cudaSuccess) return false;
+    if (cudaMalloc(&ws.counters, n_counters * sizeof(int)) != cudaSuccess) return UNSTEP_ERR_CUDA;
+    // cleared on the caller's stream, so that the clear is ordered before the kernel that follows
+    // (a non-blocking stream is not ordered against the legacy default stream)
+    if (cudaMemsetAsync(ws.counters, 0, n_counters * sizeof(int), st) != cudaSuccess) return UNSTEP_ERR_CUDA;
     ws.n_counters = n_counters;
   }
   *out = ws;
-  return true;
+  return UNSTEP_OK;
 }
 
 // After a kernel gave up, arrival counters may be left non-zero: clear them all.
@@ -955,7 +783,7 @@ using namespace unstep;
 
 // Hands out the scratch of one launch: `slots` partial-result slots and `n_counters` zeroed
 // arrival counters.
-typedef bool (*ScratchFn)(cudaStream_t st, size_t slots, size_t n_counters, Workspace* out);
+typedef int (*ScratchFn)(cudaStream_t st, size_t slots, size_t n_counters, Workspace* out);   // an unstep_status
 
 // Validation, work split, tensor maps and launch shared by the attention entry points.
 // The cache has `sink_frames` slots in front of the ring (0 for the plain rolling window);
@@ -964,20 +792,11 @@ static int window_attn_run(const unstep_shape_t* shape, const int32_t* start_fra
                            int32_t window_frames, const void* q_rot, const void* ring_k,
                            const void* ring_v, void* out, void* cuda_stream, ScratchFn scratch,
                            int32_t sink_frames = 0, int32_t sink_attend = 0) {
-  int rc = check_shape(shape, true);
+  int rc = check_attn_args(shape, start_frame, window_frames, sink_frames, sink_attend);
   if (rc != UNSTEP_OK) return rc;
-  const void* ptrs[] = {start_frame, q_rot, ring_k, ring_v, out};
+  const void* ptrs[] = {q_rot, ring_k, ring_v, out};
   for (const void* ptr : ptrs)
-    if (ptr == nullptr) return UNSTEP_ERR_INVALID_ARG;
-  if (!aligned16(q_rot) || !aligned16(ring_k) || !aligned16(ring_v) || !aligned16(out))
-    return UNSTEP_ERR_INVALID_ARG;
-  if (window_frames < shape->chunk_frames || window_frames > shape->ring_frames)
-    return UNSTEP_ERR_INVALID_ARG;
-  if (sink_frames < 0 || sink_frames > 4096 || sink_attend < 0 || sink_attend > sink_frames)
-    return UNSTEP_ERR_INVALID_ARG;
-  for (int b = 0; b < shape->batch; ++b)
-    if (start_frame[b] < 0 || start_frame[b] > INT32_MAX - shape->chunk_frames)
-      return UNSTEP_ERR_INVALID_ARG;
+    if (ptr == nullptr || !aligned16(ptr)) return UNSTEP_ERR_INVALID_ARG;
   rc = check_device();
   if (rc != UNSTEP_OK) return rc;
   const DeviceInfo& info = device_info();
@@ -988,73 +807,18 @@ static int window_attn_run(const unstep_shape_t* shape, const int32_t* start_fra
   const uint64_t T = static_cast<uint64_t>(shape->grid_h) * shape->grid_w;
   const uint64_t L = T * shape->chunk_frames;
   const uint64_t row_bytes = Hn * kHeadDim * 2;
-  if (C * T >= (uint64_t(1) << 30)) return UNSTEP_ERR_INVALID_ARG;  // cache rows are 32-bit coordinates
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
 
   AttnParams p;
-  p.sink = sink_frames;
-  p.Hn = shape->heads;
-  p.L = static_cast<int32_t>(L);
-  p.T = static_cast<int32_t>(T);
-  p.C = shape->ring_frames;
-  p.q_tiles = static_cast<int32_t>((L + kTileM - 1) / kTileM);
-  p.q_pairs = (p.q_tiles + 1) / 2;
-  p.tiles_per_frame = static_cast<int32_t>((T + kTileN - 1) / kTileN);
-  p.flat = (T >= kTileN) ? 1 : 0;  // a ragged tile must fit inside one frame
-  p.scale_log2e = 1.4426950408889634f / sqrtf(static_cast<float>(kHeadDim));
-  p.items_per_stream = p.Hn * p.q_pairs;
-
+  plan_shape(p, shape, sink_frames);
   for (int b0 = 0; b0 < shape->batch; b0 += kMaxStreamsPerLaunch) {
     const int nb = shape->batch - b0 < kMaxStreamsPerLaunch ? shape->batch - b0 : kMaxStreamsPerLaunch;
-    p.n_streams = nb;
-    for (int i = 0; i < nb; ++i) {
-      const int hi = start_frame[b0 + i] + shape->chunk_frames;
-      const int lo = hi - window_frames > 0 ? hi - window_frames : 0;
-      const int n_sink = sink_attend < lo ? sink_attend : lo;   // sink frames not already in the recent part
-      p.first_frame[i] = lo;
-      p.n_sink[i] = n_sink;
-      for (int r = 0; r < 3; ++r) p.run_row0[i][r] = p.run_rows[i][r] = p.run_tile_end[i][r] = 0;
-      if (p.flat) {
-        // walk the attended frames in order and cut them into runs of consecutive cache slots
-        int n_runs = 0, prev_slot = -2;
-        for (int k = 0; k < n_sink + hi - lo; ++k) {
-          const int frame = k < n_sink ? k : lo + k - n_sink;
-          const int slot = frame < sink_frames ? frame : sink_frames + (frame - sink_frames) % shape->ring_frames;
-          if (slot != prev_slot + 1) {
-            if (n_runs == 3) return UNSTEP_ERR_INVALID_ARG;  // cannot happen: sink, ring end, ring start
-            p.run_row0[i][n_runs++] = slot * p.T;
-          }
-          p.run_rows[i][n_runs - 1] += p.T;
-          prev_slot = slot;
-        }
-        int tiles = 0;
-        for (int r = 0; r < 3; ++r) {
-          tiles += (p.run_rows[i][r] + kTileN - 1) / kTileN;
-          p.run_tile_end[i][r] = tiles;
-        }
-        p.tiles[i] = tiles;
-      } else {
-        p.tiles[i] = (n_sink + hi - lo) * p.tiles_per_frame;
-      }
-    }
-    // grid: one CTA per SM, fewer when the whole launch is small
-    int64_t all_steps = 0;
-    for (int i = 0; i < nb; ++i)
-      all_steps += static_cast<int64_t>(p.items_per_stream) * p.tiles[i];
-    int64_t want = all_steps / kMinStepsPerCta;
-    if (want < 1) want = 1;
-    const unsigned grid = static_cast<unsigned>(want < info.sm_count ? want : info.sm_count);
-    p.full_rounds = p.items_per_stream / static_cast<int>(grid);
-    const int leftover = p.items_per_stream - p.full_rounds * static_cast<int>(grid);
-    int64_t steps = 0;
-    for (int i = 0; i < nb; ++i) {
-      p.step_base[i] = steps;
-      steps += static_cast<int64_t>(leftover) * p.tiles[i];
-    }
-    p.total_steps = steps;
+    rc = plan_launch(p, shape, start_frame + b0, nb, window_frames, sink_frames, sink_attend, info.sm_count);
+    if (rc != UNSTEP_OK) return rc;
+    const unsigned grid = static_cast<unsigned>(p.n_workers);
     Workspace ws;
-    if (!scratch(st, 2 * static_cast<size_t>(grid), 2 * static_cast<size_t>(nb) * p.items_per_stream, &ws))
-      return UNSTEP_ERR_CUDA;
+    rc = scratch(st, 2 * static_cast<size_t>(grid), 2 * static_cast<size_t>(nb) * p.items_per_stream, &ws);
+    if (rc != UNSTEP_OK) return rc;
     p.part = ws.part;
     p.counters = ws.counters;
     const char* qb = static_cast<const char*>(q_rot) + static_cast<uint64_t>(b0) * L * row_bytes;
@@ -1142,17 +906,17 @@ static unsigned char* static_scratch_base() {
 
 // Scratch source of the no-allocation entry point: carve the fixed array, clear the counters
 // this launch will use (the array keeps the previous call's contents).
-static bool static_scratch(cudaStream_t st, size_t slots, size_t n_counters, Workspace* out) {
+static int static_scratch(cudaStream_t st, size_t slots, size_t n_counters, Workspace* out) {
   if (slots > 2 * static_cast<size_t>(kStaticMaxCtas) || n_counters > static_cast<size_t>(kStaticMaxCounters))
-    return false;
+    return UNSTEP_ERR_TOO_LARGE;
   unsigned char* base = static_scratch_base();
-  if (base == nullptr) return false;
-  if (cudaMemsetAsync(base, 0, n_counters * sizeof(int), st) != cudaSuccess) return false;
+  if (base == nullptr) return UNSTEP_ERR_CUDA;
+  if (cudaMemsetAsync(base, 0, n_counters * sizeof(int), st) != cudaSuccess) return UNSTEP_ERR_CUDA;
   out->counters = reinterpret_cast<int*>(base);
   out->part = reinterpret_cast<float*>(base + kStaticCounterBytes);
   out->slots = slots;
   out->n_counters = n_counters;
-  return true;
+  return UNSTEP_OK;
 }
 
 }  // namespace unstep

@@ -41,6 +41,11 @@ class ChunkStepper:
         self.cache_v = [torch.zeros(cache, dtype=torch.bfloat16, device=self.device) for _ in range(n_layers)]
         self._tables = {}
         self._graphs = {}
+        # Every graph of this stepper is captured on this one stream.  The attention call keeps its
+        # scratch per stream and a capture freezes the scratch pointers into the graph, so one
+        # capture stream means one scratch for all graphs (replays of one stepper run one after
+        # the other on the caller's stream and may share it).
+        self._capture_stream = torch.cuda.Stream(device=self.device)
 
     def table(self, start_frame: int):
         """cos/sin of the chunk starting at `start_frame`, built once and kept (the paper's cache)."""
@@ -73,12 +78,16 @@ class ChunkStepper:
 
     def chunk_graph(self, start_frame: int, qkv, q_rot, outs):
         """A CUDA graph of chunk_step for this starting frame over these buffers (captured on
-        first use).  Replaying it re-runs every layer on whatever the buffers hold then."""
+        first use).  Replaying it re-runs every layer on whatever the buffers hold then.
+
+        The graph holds the attention scratch of the stepper's capture stream: replay the graphs of
+        a stepper one after the other (one stream), not concurrently, and capture them again after
+        `shutdown()` of the library, which frees that scratch."""
         import torch
         key = int(start_frame)
         if key not in self._graphs:
             self.table(start_frame)                  # built outside the capture
-            side = torch.cuda.Stream(device=self.device)
+            side = self._capture_stream
             side.wait_stream(torch.cuda.current_stream(self.device))
             with torch.cuda.stream(side):            # first call on this stream: scratch set-up
                 self.chunk_step(start_frame, qkv, q_rot, outs)

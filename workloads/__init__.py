@@ -95,6 +95,13 @@ WORKLOADS = {
     # window sweep, K x4, ring wrapped more than twice, measured at s=42
     "cfg3": Workload("cfg3", _S13, seed=2, history_starts=(tuple(range(0, 42, 3)),),
                      measured_starts=(42,), window_frames=(3, 6, 9, 12, 21), k_scale=4.0),
+    # second point of the sweep: measured at s=51 (slots 9..11), where only the 21-frame window wraps
+    "cfg3_s51": Workload("cfg3_s51", _S13, seed=2, history_starts=(tuple(range(0, 51, 3)),),
+                         measured_starts=(51,), window_frames=(3, 6, 9, 12, 21), k_scale=4.0),
+    # tight ring (capacity = window = 9 frames, the minimal-memory deployment), measured at s = 3*C
+    "cfg3_tight": Workload("cfg3_tight", replace(_S13, ring_frames=9), seed=2,
+                           history_starts=(tuple(range(0, 27, 3)),), measured_starts=(27,),
+                           window_frames=(9,), k_scale=4.0),
     # four streams at fill levels 0/6/12/18, clean-cache re-append pattern
     "cfg4": Workload("cfg4", replace(_S13, batch=4), seed=3,
                      history_starts=((), (0, 3), (0, 3, 6, 9), (0, 3, 6, 9, 12, 15)),
