@@ -3,7 +3,7 @@
 The chunk-attention path has no exchange step: streams (and heads) are independent, so
 N GPUs run N independent shards and nothing crosses NVLink on the data path.  What is
 shared is bookkeeping only: a barrier around the timed region, the max of a time over
-the ranks and the split of streams over ranks.  NCCL on GPUs, gloo on CPU (tests)."""
+the ranks and the split of streams or heads over ranks.  NCCL on GPUs, gloo on CPU (tests)."""
 
 from __future__ import annotations
 
@@ -65,4 +65,14 @@ def shard_streams(n_streams: int, rank: int, world: int) -> range:
     """Contiguous, balanced split of independent streams over ranks (no stream is split)."""
     lo = n_streams * rank // world
     hi = n_streams * (rank + 1) // world
+    return range(lo, hi)
+
+
+def shard_heads(n_heads: int, rank: int, world: int) -> range:
+    """Contiguous, balanced split of the attention heads over ranks.  Heads never interact, so a
+    rank that owns heads [lo, hi) keeps the cache slices [B, C, T, hi - lo, 128] of those heads,
+    appends and attends them alone, and its output is the [.., lo:hi, :] slice of the whole
+    output: no exchange inside the path (12 heads -> 2, 3, 4 or 6 GPUs; 40 heads -> 8 x 5)."""
+    lo = n_heads * rank // world
+    hi = n_heads * (rank + 1) // world
     return range(lo, hi)

@@ -124,6 +124,11 @@ WORKLOADS["cfg2_sink9_long"] = Workload("cfg2_sink9_long", replace(_S13, ring_fr
                                         window_frames=(6,), sink_frames=3, sink_attend=3)
 
 
+def with_heads(wl: Workload, heads: int) -> Workload:
+    """The same workload with another number of heads (a rank's share when heads are split over GPUs)."""
+    return replace(wl, shape=replace(wl.shape, heads=heads))
+
+
 def f32_to_bf16_bits(x: np.ndarray) -> np.ndarray:
     """Nearest-even bf16 bit pattern of finite float32 data (input generation only)."""
     u = np.ascontiguousarray(x, dtype=np.float32).view(np.uint32)
