@@ -68,7 +68,7 @@ class ClockSampler(threading.Thread):
     """Samples SM clock, power and throttle reasons of one GPU through NVML, as fast as `period_s`
     allows, with a host time stamp per sample so that a window of the run can be summarised."""
 
-    def __init__(self, index: int, period_s: float = 0.002):
+    def __init__(self, index: int, period_s: float = 0.001):
         super().__init__(daemon=True)
         self.index, self.period = index, period_s
         self.t, self.mhz, self.power, self.mask = [], [], [], []
@@ -90,11 +90,15 @@ class ClockSampler(threading.Thread):
                 getattr(nv, "nvmlClocksThrottleReasonSwPowerCap", 0x4): "sw_power_cap",
                 getattr(nv, "nvmlClocksThrottleReasonHwPowerBrakeSlowdown", 0x80): "hw_power_brake",
             }
+            n, watts = 0, 0.0
             while not self._halt.is_set():
                 self.t.append(time.perf_counter())
                 self.mhz.append(int(nv.nvmlDeviceGetClockInfo(h, nv.NVML_CLOCK_SM)))
-                self.power.append(nv.nvmlDeviceGetPowerUsage(h) / 1000.0)
+                if n % 4 == 0:                      # a query costs about a millisecond: power less often
+                    watts = nv.nvmlDeviceGetPowerUsage(h) / 1000.0
+                self.power.append(watts)
                 self.mask.append(int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(h)))
+                n += 1
                 time.sleep(self.period)
         except Exception as exc:  # NVML missing: report it, never fail the benchmark
             self.error = repr(exc)
@@ -427,18 +431,15 @@ def run_ours(args):
                      "reasons": clk_l.get("reasons"), "clock_samples": clk_l.get("samples"),
                      "mcycles_per_step": (us * clk_l["sm_mhz"] / 1e6) if clk_l.get("sm_mhz") else None}
 
-    # ---- append alone, cold (rotating sets) and warm (one set over and over) -------------
-    def append_leg(rotate, n=40):
-        ev = [torch.cuda.Event(enable_timing=True) for _ in range(n + 1)]
+    # ---- the same steps on one working set over and over: what the append gains when the lines it
+    # writes (and the attention's inputs) are still in L2 from the step before -----------------
+    def warm_leg(n=20):
+        ev = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(n)]
         for i in range(n):
-            ws = sets[(i % n_sets) if rotate else 0]
-            ev[i].record()
-            append(s, ws["q"], ws["k"], ws["v"], ws["q_rot"], ws["ring_k"], ws["ring_v"])
-        ev[n].record()
+            step(0, ev[i])
         torch.cuda.synchronize()
-        t = np.array([ev[i].elapsed_time(ev[i + 1]) for i in range(4, n)]) * 1e3
-        return float(np.median(t))
-    append_cold_us, append_warm_us = append_leg(True), append_leg(False)
+        return np.array([[e[j].elapsed_time(e[j + 1]) for j in range(3)] for e in ev[2:]]).mean(axis=0) * 1e3
+    warm_us = warm_leg()
 
     # ---- end to end: pinned host inputs in, result back to the host, every step ---------
     # Copies and kernels run on three streams with two staging buffers, so the upload of step
@@ -542,9 +543,11 @@ def run_ours(args):
                             "peak": peaks["hbm_gbs"], "unit": "GB/s",
                             "frac": append_bytes / (t_append * 1e-3) / 1e9 / peaks["hbm_gbs"],
                             "peak_source": f"{peaks['source']} copy", "bytes": append_bytes,
-                            "protocol": "inside the step, rotating working sets (cold inputs, cold outputs)",
-                            "alone_cold_us": append_cold_us, "alone_cold_frac": append_bytes / append_cold_us / 1e3 / peaks["hbm_gbs"],
-                            "alone_warm_us": append_warm_us, "alone_warm_frac": append_bytes / append_warm_us / 1e3 / peaks["hbm_gbs"]},
+                            "protocol": "timed inside the step, every step on the next working set (cold inputs, "
+                                        "cold outputs); warm_* = the same step repeated on one working set",
+                            "warm_us": float(warm_us[1]),
+                            "warm_frac": append_bytes / float(warm_us[1]) / 1e3 / peaks["hbm_gbs"],
+                            "warm_window_attn_us": float(warm_us[2])},
         "e2e": {"value": total_flops / (e2e_ms * 1e-3) / 1e12, "unit": "TFLOP/s",
                 "ms_per_step": e2e_ms, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
         "gpu_launches": int(launches), "device_status": status, "clocks": clocks,

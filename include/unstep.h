@@ -233,6 +233,14 @@ int unstep_window_attn_plan(const unstep_shape_t* shape, int32_t sink_frames, co
                             int32_t recent_frames, int32_t sink_attend, int32_t max_workers,
                             int32_t* segs, int32_t max_segs, int32_t* n_segs);
 
+/*
+ * How the attention calls will use the current device (the paper has no counterpart): the number
+ * of workers of a full-size launch (the `max_workers` to give unstep_window_attn_plan: one per SM)
+ * and the thread blocks per worker (1: every worker is one persistent thread block).
+ *   workers, ctas_per_worker : HOST int32, written.
+ */
+int unstep_attn_workers(int32_t* workers, int32_t* ctas_per_worker);
+
 /* Static, human-readable text for a status code. */
 const char* unstep_strerror(int code);
 

@@ -16,6 +16,7 @@ from .binding import (  # noqa: F401
     window_attn_sink,
     rmsnorm_rope_kv_append,
     window_attn_plan,
+    attn_workers,
     poll_status,
     shutdown,
     selftest_wait_limit,

@@ -9,7 +9,7 @@ from . import build as _build
 
 EXPORTS = ("unstep_rope_table", "unstep_rope_kv_append", "unstep_window_attn",
            "unstep_window_attn_noalloc", "unstep_rope_kv_append_sink", "unstep_window_attn_sink",
-           "unstep_rmsnorm_rope_kv_append", "unstep_window_attn_plan", "unstep_selftest_wait_limit", "unstep_shutdown", "unstep_strerror", "unstep_poll_status", "unstep_launch_count")
+           "unstep_rmsnorm_rope_kv_append", "unstep_window_attn_plan", "unstep_attn_workers", "unstep_selftest_wait_limit", "unstep_shutdown", "unstep_strerror", "unstep_poll_status", "unstep_launch_count")
 
 
 class UnstepError(RuntimeError):
@@ -75,6 +75,8 @@ def lib() -> ctypes.CDLL:
         L.unstep_window_attn_plan.restype = c_int
         L.unstep_window_attn_plan.argtypes = [POINTER(Shape), c_int32, POINTER(c_int32), c_int32, c_int32,
                                               c_int32, POINTER(c_int32), c_int32, POINTER(c_int32)]
+        L.unstep_attn_workers.restype = c_int
+        L.unstep_attn_workers.argtypes = [POINTER(c_int32), POINTER(c_int32)]
         L.unstep_selftest_wait_limit.restype = c_int
         L.unstep_selftest_wait_limit.argtypes = [c_int64, c_void_p]
         L.unstep_shutdown.restype = None
@@ -246,6 +248,13 @@ def window_attn_plan(shape: Shape, start_frame, recent_frames: int, max_workers:
     buf = (c_int32 * (10 * max(n.value, 1)))()
     _check(lib().unstep_window_attn_plan(*args, buf, n.value, ctypes.byref(n)), "unstep_window_attn_plan")
     return [tuple(buf[10 * i:10 * i + 10]) for i in range(n.value)]
+
+
+def attn_workers():
+    """unstep_attn_workers: (workers of a full-size attention launch, thread blocks per worker)."""
+    a, b = c_int32(0), c_int32(0)
+    _check(lib().unstep_attn_workers(ctypes.byref(a), ctypes.byref(b)), "unstep_attn_workers")
+    return a.value, b.value
 
 
 def selftest_wait_limit(limit_cycles: int, stream=None):

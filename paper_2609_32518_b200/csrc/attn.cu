@@ -254,6 +254,26 @@ __device__ __forceinline__ void softmax_row_tile(uint32_t t_S, uint32_t t_O, flo
   l_run += sum;
 }
 
+// Real keys of key tile j of a stream, without the divisions of tile_info: only the last tile of a
+// run of slots is ragged (frames shorter than a tile: every tile is one frame).
+struct ValidKeys {
+  int j_last[3], v_last[3], dflt;
+  __device__ __forceinline__ ValidKeys(const AttnParams& p, int b) {
+    dflt = p.flat ? kTileN : p.T;
+#pragma unroll
+    for (int r = 0; r < 3; ++r) {
+      const int begin = r == 0 ? 0 : p.run_tile_end[b][r - 1];
+      const int end = p.run_tile_end[b][r];
+      const bool any = p.flat && end > begin;
+      j_last[r] = any ? end - 1 : -1;
+      v_last[r] = p.run_rows[b][r] - kTileN * (end - begin - 1);
+    }
+  }
+  __device__ __forceinline__ int operator()(int j) const {
+    return j == j_last[0] ? v_last[0] : (j == j_last[1] ? v_last[1] : (j == j_last[2] ? v_last[2] : dflt));
+  }
+};
+
 __global__ void __launch_bounds__(kThreads, 1)
 window_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                    const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_kf,
@@ -401,7 +421,8 @@ window_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
       while (ok && sched.next(s)) {
         const bool part = a < s.nq;   // a lone last query tile leaves warp 1 only the bookkeeping
         const int n = s.t1 - s.t0;
-        int valid = tile_info(p, s.b, s.t0).valid;  // real keys of the tile S is being computed for
+        const ValidKeys valid_of(p, s.b);
+        int valid = valid_of(s.t0);  // real keys of the tile S is being computed for
         if (part) {
           ok = w.wait(bar_q_full + 8 * a, q_it & 1);
           if (!ok) break;
@@ -425,7 +446,7 @@ window_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
           ++kv_it;
           const bool more = j + 1 < n;
           if (more) {
-            valid = tile_info(p, s.b, s.t0 + j + 1).valid;
+            valid = valid_of(s.t0 + j + 1);
             kst = kv_it % kStages;
             ok = w.wait(bar_kv_full + 8 * kst, (kv_it / kStages) & 1);
             if (!ok) break;
@@ -493,8 +514,9 @@ window_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
     while (sched.next(s)) {
       if (a >= s.nq) continue;             // a lone last query tile: nothing for group 1
       float m_run = -INFINITY, l_run = 0.f;
+      const ValidKeys valid_of(p, s.b);
       for (int j = s.t0; j < s.t1 && ok; ++j) {
-        const int valid = tile_info(p, s.b, j).valid;
+        const int valid = valid_of(j);
         TRACE(a, it, 0);
         ok = w.wait(bar_s_full + 8 * a, it & 1);
         if (!ok) break;
@@ -815,9 +837,8 @@ static int window_attn_run(const unstep_shape_t* shape, const int32_t* start_fra
     const int nb = shape->batch - b0 < kMaxStreamsPerLaunch ? shape->batch - b0 : kMaxStreamsPerLaunch;
     rc = plan_launch(p, shape, start_frame + b0, nb, window_frames, sink_frames, sink_attend, info.sm_count);
     if (rc != UNSTEP_OK) return rc;
-    const unsigned grid = static_cast<unsigned>(p.n_workers);
     Workspace ws;
-    rc = scratch(st, 2 * static_cast<size_t>(grid), 2 * static_cast<size_t>(nb) * p.items_per_stream, &ws);
+    rc = scratch(st, 2 * static_cast<size_t>(p.n_workers), 2 * static_cast<size_t>(nb) * p.items_per_stream, &ws);
     if (rc != UNSTEP_OK) return rc;
     p.part = ws.part;
     p.counters = ws.counters;
@@ -837,7 +858,7 @@ static int window_attn_run(const unstep_shape_t* shape, const int32_t* start_fra
         !make_map(&tm_v, vb, 5, rdims, rstr, 2) || !make_map(&tm_kf, kb, 4, fdims, fstr, 2) ||
         !make_map(&tm_vf, vb, 4, fdims, fstr, 2))
       return UNSTEP_ERR_CUDA;
-    window_attn_kernel<<<grid, kThreads, kAttnSmemBytes, st>>>(tm_q, tm_k, tm_v, tm_kf, tm_vf, p, ob);
+    window_attn_kernel<<<p.n_workers, kThreads, kAttnSmemBytes, st>>>(tm_q, tm_k, tm_v, tm_kf, tm_vf, p, ob);
     g_launches.fetch_add(1);
     if (cudaGetLastError() != cudaSuccess) return UNSTEP_ERR_CUDA;
   }
@@ -938,6 +959,17 @@ extern "C" int unstep_window_attn_noalloc(const unstep_shape_t* shape, const int
   if (info.sm_count > kStaticMaxCtas) return UNSTEP_ERR_TOO_LARGE;
   return window_attn_run(shape, start_frame, window_frames, q_rot, ring_k, ring_v, out, cuda_stream,
                          static_scratch);
+}
+
+extern "C" int unstep_attn_workers(int32_t* workers, int32_t* ctas_per_worker) {
+  if (workers == nullptr || ctas_per_worker == nullptr) return UNSTEP_ERR_INVALID_ARG;
+  const int rc = check_device();
+  if (rc != UNSTEP_OK) return rc;
+  const DeviceInfo& info = device_info();
+  if (!info.ok) return UNSTEP_ERR_CUDA;
+  *workers = info.sm_count;
+  *ctas_per_worker = 1;
+  return UNSTEP_OK;
 }
 
 extern "C" int unstep_selftest_wait_limit(int64_t limit_cycles, void* cuda_stream) {

@@ -212,7 +212,6 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t* r) {
       "r"(r[29]), "r"(r[30]), "r"(r[31])
       : "memory");
 }
-
 // ---------------------------------------------------------------- descriptors
 // Shared-memory matrix descriptor, 128-byte swizzle (matches TMA SWIZZLE_128B).
 //   bits  0-13 start address >> 4      bits 16-29 leading byte offset >> 4
