@@ -40,7 +40,8 @@ typedef enum {
   UNSTEP_ERR_UNSUPPORTED = -2, /* head_dim != 128, device is not sm_100 */
   UNSTEP_ERR_CUDA = -3,        /* a CUDA runtime/driver call failed */
   UNSTEP_ERR_TIMEOUT = -4,     /* a bounded device-side wait expired (see unstep_poll_status) */
-  UNSTEP_ERR_TOO_LARGE = -5    /* the problem does not fit the fixed scratch of a no-allocation call */
+  UNSTEP_ERR_TOO_LARGE = -5,   /* the problem does not fit the fixed scratch of a no-allocation call */
+  UNSTEP_ERR_BOUNDS = -6       /* checking build only: a kernel tried to store outside its buffer (see below) */
 } unstep_status;
 
 typedef struct {
@@ -248,6 +249,9 @@ const char* unstep_strerror(int code);
  * Device status word of the current device: 0, or UNSTEP_ERR_TIMEOUT if a kernel gave
  * up on a bounded wait since the last poll (the word is cleared by the poll).  This
  * call synchronises the device; it is a diagnostic, not part of the hot path.
+ * In a checking build (the library compiled with -DUNSTEP_CHECK, slower) every global store of
+ * the kernels is tested against the extent of the buffer it belongs to; a store outside is
+ * skipped, never made, and the poll returns UNSTEP_ERR_BOUNDS.  Nothing traps.
  */
 int unstep_poll_status(void);
 
@@ -268,6 +272,16 @@ void unstep_shutdown(void);
 
 /* Number of kernels the library has launched in this process (all devices). */
 int64_t unstep_launch_count(void);
+
+#ifdef UNSTEP_CHECK
+/*
+ * Only in a checking build: launches one kernel whose fifth thread stores one element past the
+ * end of a 4-element range of `device_buf5` (DEVICE int32 [5]).  The store is skipped, the first
+ * four elements become 7, element 4 keeps its value and unstep_poll_status() then returns
+ * UNSTEP_ERR_BOUNDS once.  Shows that the checks are armed; nothing faults.
+ */
+int unstep_selftest_bounds_check(int32_t* device_buf5, void* cuda_stream);
+#endif
 
 #ifdef UNSTEP_TRACE
 /*

@@ -47,7 +47,8 @@ def lib() -> ctypes.CDLL:
     """Load (building first if stale) the CUDA library; raises if that is impossible."""
     global _lib
     if _lib is None:
-        path = _build.build()
+        import os
+        path = _build.build(variant=os.environ.get("UNSTEP_LIB_VARIANT", ""))
         L = ctypes.CDLL(path)
         L.unstep_rope_table.restype = c_int
         L.unstep_rope_table.argtypes = [POINTER(Shape), c_int32, c_void_p, c_void_p, c_void_p]

@@ -29,27 +29,44 @@ def _inputs():
     return files
 
 
-def is_stale() -> bool:
-    if not os.path.exists(LIB_PATH):
+# Diagnostic variants of the library, built beside the normal one as libunstep_<name>.so and
+# loaded instead of it when the environment variable UNSTEP_LIB_VARIANT names one.
+VARIANTS = {
+    "check": ["-DUNSTEP_CHECK"],   # every global store bounds-checked, violations reported, never made
+}
+
+
+def lib_path(variant: str = "") -> str:
+    return LIB_PATH if not variant else os.path.join(PKG_DIR, f"libunstep_{variant}.so")
+
+
+def is_stale(variant: str = "") -> bool:
+    path = lib_path(variant)
+    if not os.path.exists(path):
         return True
-    built = os.path.getmtime(LIB_PATH)
+    built = os.path.getmtime(path)
     return any(os.path.getmtime(f) > built for f in _inputs())
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
-    """Compile the library if it is missing or older than its sources; return its path."""
-    if not force and not is_stale():
-        return LIB_PATH
+def build(force: bool = False, verbose: bool = False, variant: str = "") -> str:
+    """Compile the library (or a diagnostic variant of it) if it is missing or older than its
+    sources; return its path."""
+    if variant and variant not in VARIANTS:
+        raise ValueError(f"unknown library variant {variant!r}")
+    path = lib_path(variant)
+    if not force and not is_stale(variant):
+        return path
     extra = os.environ.get("UNSTEP_NVCC_FLAGS", "").split()  # e.g. -DUNSTEP_TRACE for a debug build
+    extra += VARIANTS.get(variant, [])
     cmd = [_nvcc()] + NVCC_FLAGS + extra + (["-Xptxas", "-v"] if verbose else []) + [
-        "-I", INCLUDE, "-I", CSRC, "-o", LIB_PATH + ".tmp"] + [os.path.join(CSRC, s) for s in SOURCES]
+        "-I", INCLUDE, "-I", CSRC, "-o", path + ".tmp"] + [os.path.join(CSRC, s) for s in SOURCES]
     res = subprocess.run(cmd, capture_output=True, text=True)
     if res.returncode != 0:
         raise RuntimeError("nvcc failed:\n" + res.stdout + res.stderr)
-    os.replace(LIB_PATH + ".tmp", LIB_PATH)
+    os.replace(path + ".tmp", path)
     if verbose:
         print(res.stderr)
-    return LIB_PATH
+    return path
 
 
 if __name__ == "__main__":

@@ -14,6 +14,7 @@ extern "C" const char* unstep_strerror(int code) {
     case UNSTEP_ERR_CUDA: return "a CUDA call failed";
     case UNSTEP_ERR_TIMEOUT: return "a bounded device-side wait expired";
     case UNSTEP_ERR_TOO_LARGE: return "too large for the fixed scratch of the no-allocation entry point";
+    case UNSTEP_ERR_BOUNDS: return "checking build: a kernel tried to store outside its buffer (the store was skipped)";
     default: return "unknown status";
   }
 }

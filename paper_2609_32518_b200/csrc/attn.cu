@@ -537,9 +537,9 @@ window_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         tc_fence_after();
       }
       const int n = (2 * s.qp + a) * kTileM + row;
-      uint4* dst = reinterpret_cast<uint4*>(
-          out + ((static_cast<int64_t>(s.b) * p.L + n) * p.Hn + s.h) * kHeadDim);
-      auto store_row = [&](uint4* d, const float* v, float inv_l) {   // 32 columns
+      uint4* const out_v = reinterpret_cast<uint4*>(out);
+      const int64_t dst = ((static_cast<int64_t>(s.b) * p.L + n) * p.Hn + s.h) * (kHeadDim / 8);   // 16-byte vectors
+      auto store_row = [&](int64_t d, const float* v, float inv_l) {   // 32 columns from vector d on
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
           uint4 vv;
@@ -547,7 +547,7 @@ window_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
           vv.y = pack_bf16x2(v[8 * i + 2] * inv_l, v[8 * i + 3] * inv_l);
           vv.z = pack_bf16x2(v[8 * i + 4] * inv_l, v[8 * i + 5] * inv_l);
           vv.w = pack_bf16x2(v[8 * i + 6] * inv_l, v[8 * i + 7] * inv_l);
-          d[i] = vv;
+          UNSTEP_STORE(out_v, d + i, p.extent_out, vv, p.status);
         }
       };
       const bool whole = (s.t0 == 0 && s.t1 == s.tiles);
@@ -574,6 +574,9 @@ window_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         const int c_hi = last_part_worker(p, s);
         const int others = c_hi - c_lo;
         int* counter = p.counters + 2 * s.item + a;
+#ifdef UNSTEP_CHECK
+        if (row == 0 && 2 * s.item + a >= p.extent_counters) atomicExch(p.status, static_cast<int>(UNSTEP_ERR_BOUNDS));
+#endif
         if (row == 0 && ok) {
           int seen;
           asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(seen) : "l"(counter) : "memory");
@@ -583,18 +586,19 @@ window_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         if (*abort_flag) break;            // raised before the barrier by whoever gave up
         bool last = (*my_flag != 0);
         if (!last) {
-          float* mine = p.part + (static_cast<int64_t>(2 * blockIdx.x + (s.first_in_worker ? 0 : 1)) * kPartFloats +
-                                  a * kPartTileFloats);
+          const int64_t mine = static_cast<int64_t>(2 * blockIdx.x + (s.first_in_worker ? 0 : 1)) * kPartFloats +
+                               a * kPartTileFloats;   // first float of this part in the scratch
 #pragma unroll
           for (int q = 0; q < 4; ++q) {
             uint32_t o[32];
             tmem_ld32(t_O + q * 32, o);
             tc_wait_ld32(o);
 #pragma unroll
-            for (int i = 0; i < 32; ++i) mine[(q * 32 + i) * 128 + row] = __uint_as_float(o[i]);
+            for (int i = 0; i < 32; ++i)
+              UNSTEP_STORE(p.part, mine + (q * 32 + i) * 128 + row, p.extent_part, __uint_as_float(o[i]), p.status);
           }
-          mine[128 * 128 + row] = m_run;
-          mine[128 * 128 + 128 + row] = l_run;
+          UNSTEP_STORE(p.part, mine + 128 * 128 + row, p.extent_part, m_run, p.status);
+          UNSTEP_STORE(p.part, mine + 128 * 128 + 128 + row, p.extent_part, l_run, p.status);
           __threadfence();
           group_barrier(a);   // all of this part is published; everyone has read the flag
           if (row == 0) {
@@ -610,7 +614,7 @@ window_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         }
         if (last) {
           __threadfence();   // acquire side for every thread that reads the other parts below
-          if (row == 0) *counter = 0;   // ready for the next launch
+          if (row == 0) UNSTEP_STORE(p.counters, 2 * s.item + a, p.extent_counters, 0, p.status);   // ready for the next launch
           const int me = static_cast<int>(blockIdx.x);
           auto part_of = [&](int c) -> const float* {
             return p.part + (static_cast<int64_t>(2 * c + part_slot(p, c, s.item_step0)) * kPartFloats +
@@ -799,6 +803,21 @@ static void reset_workspace_counters() {
       cudaMemset(kv.second.counters, 0, kv.second.n_counters * sizeof(int));
 }
 
+// Device address of g_status on the current device, looked up once per device.
+int* status_word() {
+  static std::mutex mutex;
+  static int* addr[64] = {};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+  std::lock_guard<std::mutex> lock(mutex);
+  if (addr[dev] == nullptr) {
+    void* ptr = nullptr;
+    if (cudaGetSymbolAddress(&ptr, g_status) != cudaSuccess) return nullptr;
+    addr[dev] = static_cast<int*>(ptr);
+  }
+  return addr[dev];
+}
+
 }  // namespace unstep
 
 using namespace unstep;
@@ -842,6 +861,10 @@ static int window_attn_run(const unstep_shape_t* shape, const int32_t* start_fra
     if (rc != UNSTEP_OK) return rc;
     p.part = ws.part;
     p.counters = ws.counters;
+    p.status = status_word();
+    p.extent_out = static_cast<int64_t>(nb) * p.L * p.Hn * (kHeadDim / 8);
+    p.extent_part = static_cast<int64_t>(ws.slots) * kPartFloats;
+    p.extent_counters = static_cast<int64_t>(ws.n_counters);
     const char* qb = static_cast<const char*>(q_rot) + static_cast<uint64_t>(b0) * L * row_bytes;
     const char* kb = static_cast<const char*>(ring_k) + static_cast<uint64_t>(b0) * C * T * row_bytes;
     const char* vb = static_cast<const char*>(ring_v) + static_cast<uint64_t>(b0) * C * T * row_bytes;
@@ -972,6 +995,26 @@ extern "C" int unstep_attn_workers(int32_t* workers, int32_t* ctas_per_worker) {
   return UNSTEP_OK;
 }
 
+#ifdef UNSTEP_CHECK
+namespace unstep {
+// One store just past the end of a 4-element buffer: a checking build must skip it and record it.
+__global__ void check_probe_kernel(int* buf, int* status) {
+  UNSTEP_STORE(buf, threadIdx.x, 4, 7, status);
+}
+}  // namespace unstep
+
+extern "C" int unstep_selftest_bounds_check(int32_t* device_buf5, void* cuda_stream) {
+  if (device_buf5 == nullptr) return UNSTEP_ERR_INVALID_ARG;
+  const int rc = check_device();
+  if (rc != UNSTEP_OK) return rc;
+  int* st = status_word();
+  if (st == nullptr) return UNSTEP_ERR_CUDA;
+  check_probe_kernel<<<1, 5, 0, static_cast<cudaStream_t>(cuda_stream)>>>(device_buf5, st);
+  g_launches.fetch_add(1);
+  return cudaGetLastError() == cudaSuccess ? UNSTEP_OK : UNSTEP_ERR_CUDA;
+}
+#endif
+
 extern "C" int unstep_selftest_wait_limit(int64_t limit_cycles, void* cuda_stream) {
   if (limit_cycles < 1 || limit_cycles > 4000000000LL) return UNSTEP_ERR_INVALID_ARG;
   const int rc = check_device();
@@ -1003,7 +1046,7 @@ extern "C" int unstep_poll_status(void) {
   if (cudaMemcpyFromSymbol(&st, g_status, sizeof(int)) != cudaSuccess) return UNSTEP_ERR_CUDA;
   if (st != 0) {
     if (cudaMemcpyToSymbol(g_status, &zero, sizeof(int)) != cudaSuccess) return UNSTEP_ERR_CUDA;
-    reset_workspace_counters();
+    if (st == UNSTEP_ERR_TIMEOUT) reset_workspace_counters();
   }
   return st;
 }

@@ -36,6 +36,10 @@ struct AttnParams {
   int64_t total_steps;      // remainder: sum over the leftover items of their key tiles
   float* part;              // workspace: partial results of split items, kPartFloats per slot
   int* counters;            // workspace: arrivals per (item, query tile), zero between launches
+  int* status;              // status word; with the extents below, for checking builds
+  int64_t extent_out;       // 16-byte vectors of `out` that belong to this launch's streams
+  int64_t extent_part;      // floats of `part`
+  int64_t extent_counters;  // ints of `counters`
   int32_t sink;             // S: cache slots [0, S) hold frames [0, S) for good, the ring follows
   int32_t first_frame[kMaxStreamsPerLaunch];  // first frame of the recent part of stream b
   int32_t n_sink[kMaxStreamsPerLaunch];       // sink frames attended in front of the recent part
@@ -254,6 +258,8 @@ inline void plan_shape(AttnParams& p, const unstep_shape_t* shape, int32_t sink_
   p.items_per_stream = p.Hn * p.q_pairs;
   p.part = nullptr;
   p.counters = nullptr;
+  p.status = nullptr;
+  p.extent_out = p.extent_part = p.extent_counters = 0;
 }
 
 // Argument checks shared by the attention entry points and the plan entry point (no device needed).

@@ -16,6 +16,24 @@ constexpr int kMaxStreamsPerLaunch = 32;  // per-stream host scalars travel as k
 
 extern std::atomic<int64_t> g_launches;
 
+// Device address of the status word on the current device (null if it cannot be found).
+int* status_word();
+
+// A checking build (-DUNSTEP_CHECK) tests every global store of the kernels against the extent of
+// the buffer it belongs to; a store outside is skipped and recorded in the status word (no trap),
+// so that a wrong index shows up as UNSTEP_ERR_BOUNDS instead of silent corruption.  This stands
+// in for a memory checker where none can be run.  In a normal build the macro is the plain store.
+#ifdef UNSTEP_CHECK
+#define UNSTEP_STORE(base, idx, extent, value, status)                                  \
+  do {                                                                                  \
+    const long long idx_ = static_cast<long long>(idx);                                 \
+    if (idx_ >= 0 && idx_ < static_cast<long long>(extent)) (base)[idx_] = (value);     \
+    else atomicExch((status), static_cast<int>(UNSTEP_ERR_BOUNDS));                     \
+  } while (0)
+#else
+#define UNSTEP_STORE(base, idx, extent, value, status) ((base)[idx] = (value))
+#endif
+
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 // Shape checks common to every call.  `need_ring` also checks batch/heads/ring_frames.

@@ -13,6 +13,8 @@ struct TableParams {
   int32_t pairs_t, pairs_h;  // pairs_w = 64 - pairs_t - pairs_h
   int32_t band_t, band_h, band_w;
   double base;
+  int* status;       // status word and extent (floats) of each output, for checking builds
+  int64_t extent;
 };
 
 // cos and sin of position * omega in double, rounded once.
@@ -60,8 +62,8 @@ __global__ void __launch_bounds__(1024) rope_table_kernel(TableParams p, float* 
     for (int idx = threadIdx.x; idx < cols * kPairs; idx += blockDim.x) {
       const int c = idx >> 6, j = idx & 63;
       const float2 v = j < n_fixed ? band[j] : band[n_fixed + c * pairs_w + (j - n_fixed)];
-      cos_out[row_base + c0 * kPairs + idx] = v.x;
-      sin_out[row_base + c0 * kPairs + idx] = v.y;
+      UNSTEP_STORE(cos_out, row_base + c0 * kPairs + idx, p.extent, v.x, p.status);
+      UNSTEP_STORE(sin_out, row_base + c0 * kPairs + idx, p.extent, v.y, p.status);
     }
     __syncthreads();
   }
@@ -78,6 +80,8 @@ struct AppendParams {
   int64_t ring_vec_per_stream;     // (S + C) * T * Hn * 16
   int64_t table_stream_stride;     // elements
   int32_t start[kMaxStreamsPerLaunch];  // start_frame[b]
+  int* status;                     // status word and extents (16-byte vectors) of q_out and of the cache
+  int64_t extent_act, extent_cache;     // of this launch's streams, for checking builds
 };
 
 __device__ __forceinline__ uint32_t rotate_pair(uint32_t w, float c, float s) {
@@ -125,9 +129,9 @@ rope_kv_append_kernel(AppendParams p, const uint4* q_in, const uint4* __restrict
 
   const int64_t ring_idx = static_cast<int64_t>(b) * p.ring_vec_per_stream +
                            (static_cast<int64_t>(slot) * p.T + t) * p.vec_per_token + rem;
-  q_out[in_idx] = rotate_vec(xq, c, s);
-  ring_k[ring_idx] = rotate_vec(xk, c, s);
-  ring_v[ring_idx] = xv;
+  UNSTEP_STORE(q_out, in_idx, p.extent_act, rotate_vec(xq, c, s), p.status);
+  UNSTEP_STORE(ring_k, ring_idx, p.extent_cache, rotate_vec(xk, c, s), p.status);
+  UNSTEP_STORE(ring_v, ring_idx, p.extent_cache, xv, p.status);
 }
 
 // --------------------------------------------------------------------------
@@ -229,9 +233,9 @@ rmsnorm_rope_kv_append_kernel(AppendParams p, float eps, const uint4* q_in, cons
     const float4 s = __ldg(sin_t + tab_base + (vi & 15));
     const uint4 nq = normalise_vec(xq, rq, __ldg(gain_q + 2 * vi), __ldg(gain_q + 2 * vi + 1));
     const uint4 nk = normalise_vec(xk, rk, __ldg(gain_k + 2 * vi), __ldg(gain_k + 2 * vi + 1));
-    q_out[in_base + vi] = rotate_vec(nq, c, s);
-    ring_k[ring_base + vi] = rotate_vec(nk, c, s);
-    ring_v[ring_base + vi] = __ldcs(v_in + in_base + vi);
+    UNSTEP_STORE(q_out, in_base + vi, p.extent_act, rotate_vec(nq, c, s), p.status);
+    UNSTEP_STORE(ring_k, ring_base + vi, p.extent_cache, rotate_vec(nk, c, s), p.status);
+    UNSTEP_STORE(ring_v, ring_base + vi, p.extent_cache, __ldcs(v_in + in_base + vi), p.status);
   };
   {
     for (int v0 = lane; v0 < p.vec_per_token; v0 += 32 * 2) {
@@ -274,6 +278,8 @@ extern "C" int unstep_rope_table(const unstep_shape_t* shape, int32_t start_fram
   p.band_h = shape->band_h;
   p.band_w = shape->band_w;
   p.base = shape->rope_base;
+  p.status = status_word();
+  p.extent = static_cast<int64_t>(p.L) * kPairs;
   if (shape->chunk_frames > 65535) return UNSTEP_ERR_INVALID_ARG;
   rope_table_kernel<<<dim3(shape->grid_h, shape->chunk_frames), 1024, 0,
                       static_cast<cudaStream_t>(cuda_stream)>>>(p, cos_out, sin_out);
@@ -317,6 +323,9 @@ static int rope_kv_append_run(const unstep_shape_t* shape, int32_t sink_frames,
   for (int b0 = 0; b0 < shape->batch; b0 += kMaxStreamsPerLaunch) {
     const int nb = shape->batch - b0 < kMaxStreamsPerLaunch ? shape->batch - b0 : kMaxStreamsPerLaunch;
     for (int i = 0; i < nb; ++i) p.start[i] = start_frame[b0 + i];
+    p.status = status_word();
+    p.extent_act = nb * p.vec_per_stream;
+    p.extent_cache = nb * p.ring_vec_per_stream;
     const int64_t in_off = static_cast<int64_t>(b0) * p.vec_per_stream;
     const int64_t ring_off = static_cast<int64_t>(b0) * p.ring_vec_per_stream;
     const int64_t tab_off = static_cast<int64_t>(b0) * table_stream_stride;
@@ -386,6 +395,9 @@ extern "C" int unstep_rmsnorm_rope_kv_append(const unstep_shape_t* shape, int32_
   for (int b0 = 0; b0 < shape->batch; b0 += kMaxStreamsPerLaunch) {
     const int nb = shape->batch - b0 < kMaxStreamsPerLaunch ? shape->batch - b0 : kMaxStreamsPerLaunch;
     for (int i = 0; i < nb; ++i) p.start[i] = start_frame[b0 + i];
+    p.status = status_word();
+    p.extent_act = nb * p.vec_per_stream;
+    p.extent_cache = nb * p.ring_vec_per_stream;
     const int64_t in_off = static_cast<int64_t>(b0) * p.vec_per_stream;
     const int64_t ring_off = static_cast<int64_t>(b0) * p.ring_vec_per_stream;
     const int64_t tab_off = static_cast<int64_t>(b0) * table_stream_stride;

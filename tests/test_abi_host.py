@@ -19,7 +19,7 @@ def declared_functions():
     for fn in os.listdir(os.path.join(ROOT, "include")):
         text = open(os.path.join(ROOT, "include", fn)).read()
         text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
-        text = re.sub(r"#ifdef UNSTEP_TRACE.*?#endif", "", text, flags=re.S)   # diagnostic builds only
+        text = re.sub(r"#ifdef UNSTEP_(TRACE|CHECK).*?#endif", "", text, flags=re.S)   # diagnostic builds only
         names |= set(re.findall(r"\b(unstep_[a-z0-9_]+)\s*\(", text))
     return names
 
