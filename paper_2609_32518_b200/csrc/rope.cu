@@ -137,7 +137,11 @@ rope_kv_append_kernel(AppendParams p, const uint4* q_in, const uint4* __restrict
 // --------------------------------------------------------------------------
 // RMSNorm of q and k fused in front of the rotation: one warp per token.  The norm runs over
 // the whole token vector (all heads).  Pass 1 loads the token's q and k vectors and sums their
-// squares in double (exact for bf16 data, so the order of summation does not matter); pass 2
+// squares in double.  Each square is exact; the additions round at 2^-53 relative, so a sum taken
+// in another order than the reference's can differ from it in the last bits of the double (and
+// not at all unless the squares of one token span more than about 2^26 in magnitude), far below
+// the rounding of the mean to float32 that follows: the float32 mean, and with it every output
+// bit, does not depend on the order except in a near-tie of that rounding.  Pass 2
 // normalises (float32: sqrt, reciprocal and two products, each rounded once), rounds to bf16 as
 // the unfused pipeline would, rotates and stores.  Pass 2 reads q and k again, from L1/L2:
 // keeping them in registers between the passes cost more in occupancy than the second read.
@@ -148,22 +152,25 @@ __device__ __forceinline__ double warp_sum(double x) {
   for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xFFFFFFFFu, x, o);
   return x;
 }
-// Exact widening of a non-negative float to double with integer operations (the conversion
-// instruction is a slow-rate one): rebias the exponent, move the mantissa.  Zero and float
-// denormals take the ordinary conversion.
-__device__ __forceinline__ double widen_nonneg(float v) {
-  const uint32_t u = __float_as_uint(v);
-  if ((u & 0x7F800000u) == 0u) return static_cast<double>(v);
-  return __hiloint2double(static_cast<int>((u >> 3) + 0x38000000u), static_cast<int>(u << 29));
+// |x| of a bf16 as a double, built with integer operations (sign dropped: only squares are
+// formed): the 8 exponent bits are rebiased into the double's exponent field, the 7 mantissa bits
+// land at its top.  `hi_word_bits` holds the bf16's exponent and mantissa at bits 27..13.
+// Zero and bf16 denormals come out as about 2^-127 instead: their squares (below 2^-252) vanish
+// when the mean is rounded to float32, exactly as the true ones do.
+__device__ __forceinline__ double abs_bf16_as_double(uint32_t hi_word_bits) {
+  return __hiloint2double(static_cast<int>((hi_word_bits & 0x0FFFE000u) + 0x38000000u), 0);
 }
-__device__ __forceinline__ double squares(uint4 x) {
-  double s0 = 0.0, s1 = 0.0;
+// Sum of the squares of the 8 bf16 of a vector, in double.  A bf16 square has 16 significant
+// bits, so each fused multiply-add adds an exact square and rounds once, like the additions of
+// the reference's double-precision sum.
+__device__ __forceinline__ double squares(uint4 x, double acc) {
+  double s0 = acc, s1 = 0.0;
   const uint32_t w[4] = {x.x, x.y, x.z, x.w};
 #pragma unroll
   for (int i = 0; i < 4; ++i) {
-    const float lo = __uint_as_float(w[i] << 16), hi = __uint_as_float(w[i] & 0xFFFF0000u);
-    s0 += widen_nonneg(lo * lo);   // a bf16 square has 16 significant bits: exact in float
-    s1 += widen_nonneg(hi * hi);
+    const double lo = abs_bf16_as_double(w[i] << 13), hi = abs_bf16_as_double(w[i] >> 3);
+    s0 = fma(lo, lo, s0);
+    s1 = fma(hi, hi, s1);
   }
   return s0 + s1;
 }
@@ -217,8 +224,8 @@ rmsnorm_rope_kv_append_kernel(AppendParams p, float eps, const uint4* q_in, cons
 #pragma unroll
       for (int u = 0; u < 4; ++u) {
         if (v0 + 32 * u < p.vec_per_token) {
-          sq += squares(xq[u]);
-          sk += squares(xk[u]);
+          sq = squares(xq[u], sq);
+          sk = squares(xk[u], sk);
         }
       }
     }

@@ -37,7 +37,18 @@ def _full_compare(request):
 
 
 FULL = False
-ERRORS = {}   # (workload, window) -> (max abs, mean abs, relative L2, "full" or "sampled"), for reports
+ERRORS = {}   # (workload, window, pass) -> (max abs, mean abs, relative L2, "full" or "sampled"), for reports
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _error_report():
+    """UNSTEP_ERRORS_JSON=<path>: write the measured errors of this module's comparisons there."""
+    yield
+    path = os.environ.get("UNSTEP_ERRORS_JSON")
+    if path and ERRORS:
+        import json
+        with open(path, "w") as fh:
+            json.dump({f"{k[0]} Wf={k[1]} pass={k[2]}": v for k, v in ERRORS.items()}, fh, indent=1)
 
 
 def run(wl, rows_fn=None, heads=None, tag=0, dev=None, ora=None):
