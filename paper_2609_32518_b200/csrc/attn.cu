@@ -435,6 +435,9 @@ window_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         if (part) {
           tc_fence_after();
           issue_qk(kst, valid);
+          // Q is free as soon as the item's last Q K^T has run: the producer fetches the next
+          // item's Q under this item's last exponentials and P V
+          if (n == 1) tc_commit(bar_q_empty + 8 * a);
         } else {
           mbar_arrive(bar_kv_empty + 8 * kst);
         }
@@ -472,6 +475,7 @@ window_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
             TRACE(2 + a, sp_it, 4);
             // the next S first (it is what the softmax warps wait for), the stage releases after it
             if (more) issue_qk(kst, valid);
+            if (j + 2 == n) tc_commit(bar_q_empty + 8 * a);
             tc_commit(bar_kv_empty + 8 * vst);
             if (s.nq == 2) {
               mbar_arrive(bar_mturn + 8 * (1 - a));
@@ -485,10 +489,7 @@ window_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
           }
         }
         if (!ok) break;
-        if (part) {
-          tc_commit(bar_o_final + 8 * a);
-          tc_commit(bar_q_empty + 8 * a);
-        }
+        if (part) tc_commit(bar_o_final + 8 * a);
       }
     }
   } else {

@@ -20,11 +20,25 @@ pytestmark = pytest.mark.gpu
 MAX_ABS, MEAN_ABS, REL_L2 = 2e-2, 2e-3, 1.5e-2
 
 
-def check(got_bits, ref, what=""):
+# Workloads whose keys are scaled have outputs of magnitude 4 and more (a peaked softmax returns
+# single value rows).  There the rounding of the bf16 RESULT alone is up to half a unit in the last
+# place = 2^-8 |o| = 1.56e-2 at |o| = 4, which leaves an ideal bf16-P / bf16-out pipeline no room
+# under an absolute 2e-2 on every one of millions of elements.  The named configurations keep the
+# absolute bound on every element; the extra stress shapes bound each element by
+# max(2e-2, 1.5 * 2^-8 |reference|): one rounding of the result plus half as much for the rounding
+# of P, whose relative error is 2^-9 per weight.
+STRICT = {"cfg1", "cfg1_wrapped", "cfg2", "cfg3", "cfg3_s51", "cfg4", "cfg5"}
+
+
+def check(got_bits, ref, what="", strict=True):
     mx, mean, rel = attn_errors(got_bits, ref)
-    assert np.isfinite(O.bf16_bits_to_f32(got_bits)).all(), f"{what}: non-finite output"
-    assert mx <= MAX_ABS and mean <= MEAN_ABS and rel <= REL_L2, \
-        f"{what}: max {mx:.3e} mean {mean:.3e} relL2 {rel:.3e}"
+    got = O.bf16_bits_to_f32(got_bits).astype(np.float64)
+    assert np.isfinite(got).all(), f"{what}: non-finite output"
+    if strict:
+        ok_max = mx <= MAX_ABS
+    else:
+        ok_max = bool((np.abs(got - ref) <= np.maximum(MAX_ABS, 1.5 * 2.0 ** -8 * np.abs(ref))).all())
+    assert ok_max and mean <= MEAN_ABS and rel <= REL_L2, f"{what}: max {mx:.3e} mean {mean:.3e} relL2 {rel:.3e}"
     return mx, mean, rel
 
 
@@ -74,7 +88,7 @@ def run(wl, rows_fn=None, heads=None, tag=0, dev=None, ora=None):
         got = out if rows is None else out[:, rows]
         if heads is not None:
             got = got[:, :, heads]
-        ERRORS[(wl.name, wf, tag)] = check(got, ref, f"{wl.name} Wf={wf}") + ("full" if rows is None and heads is None else "sampled",)
+        ERRORS[(wl.name, wf, tag)] = check(got, ref, f"{wl.name} Wf={wf}", strict=wl.name in STRICT) + ("full" if rows is None and heads is None else "sampled",)
     assert U.poll_status() == 0
     return dev, ora
 
