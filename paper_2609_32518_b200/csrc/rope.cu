@@ -189,6 +189,10 @@ __device__ __forceinline__ uint4 normalise_vec(uint4 x, float r, float4 g0, floa
   return make_uint4(y[0], y[1], y[2], y[3]);
 }
 
+// kVFirst: the V copy rides along with pass 1, so that its traffic overlaps the wait for q and k.
+// It costs 13 registers (74 instead of 61): worth it when the tokens need several waves of warps
+// anyway (14B shape: 165 -> 152 us), not when they just fit one wave (1.3B shape: 23.8 -> 25.3 us).
+template <bool kVFirst>
 __global__ void __launch_bounds__(256)
 rmsnorm_rope_kv_append_kernel(AppendParams p, float eps, const uint4* q_in, const uint4* __restrict__ k_in,
                               const uint4* __restrict__ v_in, const float4* __restrict__ gain_q,
@@ -213,12 +217,14 @@ rmsnorm_rope_kv_append_kernel(AppendParams p, float eps, const uint4* q_in, cons
     // four vectors of q and of k per lane in flight at a time
     for (int v0 = lane; v0 < p.vec_per_token; v0 += 32 * 4) {
       uint4 xq[4], xk[4];
+      uint4 xv[4];
 #pragma unroll
       for (int u = 0; u < 4; ++u) {
         const int vi = v0 + 32 * u;
         if (vi < p.vec_per_token) {
           xq[u] = q_in[in_base + vi];   // plain load: q_out may be the same buffer
           xk[u] = __ldg(k_in + in_base + vi);
+          if (kVFirst) xv[u] = __ldcs(v_in + in_base + vi);
         }
       }
 #pragma unroll
@@ -226,6 +232,7 @@ rmsnorm_rope_kv_append_kernel(AppendParams p, float eps, const uint4* q_in, cons
         if (v0 + 32 * u < p.vec_per_token) {
           sq = squares(xq[u], sq);
           sk = squares(xk[u], sk);
+          if (kVFirst) UNSTEP_STORE(ring_v, ring_base + v0 + 32 * u, p.extent_cache, xv[u], p.status);
         }
       }
     }
@@ -242,7 +249,7 @@ rmsnorm_rope_kv_append_kernel(AppendParams p, float eps, const uint4* q_in, cons
     const uint4 nk = normalise_vec(xk, rk, __ldg(gain_k + 2 * vi), __ldg(gain_k + 2 * vi + 1));
     UNSTEP_STORE(q_out, in_base + vi, p.extent_act, rotate_vec(nq, c, s), p.status);
     UNSTEP_STORE(ring_k, ring_base + vi, p.extent_cache, rotate_vec(nk, c, s), p.status);
-    UNSTEP_STORE(ring_v, ring_base + vi, p.extent_cache, __ldcs(v_in + in_base + vi), p.status);
+    if (!kVFirst) UNSTEP_STORE(ring_v, ring_base + vi, p.extent_cache, __ldcs(v_in + in_base + vi), p.status);
   };
   {
     for (int v0 = lane; v0 < p.vec_per_token; v0 += 32 * 2) {
@@ -418,7 +425,14 @@ extern "C" int unstep_rmsnorm_rope_kv_append(const unstep_shape_t* shape, int32_
     uint4* qo = static_cast<uint4*>(q_out) + in_off;
     uint4* rk = static_cast<uint4*>(cache_k) + ring_off;
     uint4* rv = static_cast<uint4*>(cache_v) + ring_off;
-    rmsnorm_rope_kv_append_kernel<<<dim3(blocks, nb), 256, 0, st>>>(p, eps, q, k, v, gq, gk, ct, sn, qo, rk, rv);
+    // one warp per token: beyond about 32 resident warps per SM the tokens run in waves
+    int sms = 148;
+    int dev = 0;
+    if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    if (static_cast<int64_t>(nb) * L > static_cast<int64_t>(sms) * 32)
+      rmsnorm_rope_kv_append_kernel<true><<<dim3(blocks, nb), 256, 0, st>>>(p, eps, q, k, v, gq, gk, ct, sn, qo, rk, rv);
+    else
+      rmsnorm_rope_kv_append_kernel<false><<<dim3(blocks, nb), 256, 0, st>>>(p, eps, q, k, v, gq, gk, ct, sn, qo, rk, rv);
     g_launches.fetch_add(1);
     if (cudaGetLastError() != cudaSuccess) return UNSTEP_ERR_CUDA;
   }
