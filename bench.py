@@ -163,23 +163,34 @@ def oracle_sample(wl, heads, rows_per_head, repeats=1):
     return dt, flops, desc
 
 
+def reference_sample_size(steps: int, warmup: int):
+    """(heads, query rows per head) of one reference step: the largest sample of the table whose
+    steps + warmup repetitions stay near two and a half minutes on a few host cores."""
+    per_step = 150.0 / max(1, steps + warmup)
+    for seconds, heads, rows in ((8.0, 2, 2340), (4.0, 1, 2340), (2.0, 1, 1024)):
+        if per_step >= seconds:
+            return heads, rows
+    return 1, 256
+
+
 def run_reference(args):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
     wl = W.WORKLOADS[WORKLOAD]
     cores = len(os.sched_getaffinity(0))
-    oracle_sample(wl, 1, 256)  # warm numpy/BLAS
-    for _ in range(max(0, min(args.warmup, 1))):
-        oracle_sample(wl, 1, 1024)
+    steps, warmup = max(1, args.steps), max(0, args.warmup)
+    heads, rows = reference_sample_size(steps, warmup)
+    for _ in range(warmup):
+        oracle_sample(wl, heads, rows)
     times, flops, desc = [], 0.0, ""
-    for _ in range(max(1, min(args.steps, 3))):
-        dt, flops, desc = oracle_sample(wl, 2, 2340)
+    for _ in range(steps):
+        dt, flops, desc = oracle_sample(wl, heads, rows)
         times.append(dt)
     dt = float(np.mean(times))
     val = flops / dt / 1e12
     line = {"impl": "reference", "metric": METRIC, "value": val, "unit": "TFLOP/s", "n_gpus": args.gpus,
-            "steps": len(times), "warmup": min(args.warmup, 1), "ms_per_step": dt * 1e3,
+            "steps": steps, "warmup": warmup, "ms_per_step": dt * 1e3,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
             "data": "synthetic", "config": {"workload": WORKLOAD, "sample": desc},
             "cpu_baseline": {"value": val, "unit": "TFLOP/s", "cores": cores, "kind": "oracle",
