@@ -550,7 +550,7 @@ def run_ours(args):
                      "traffic_source": ATTN_DRAM_TRAFFIC if default_cfg else None,
                      "mcycles_per_launch": (t_attn * 1e3 * clocks["sm_mhz"] / 1e6) if clocks and clocks.get("sm_mhz") else None,
                      "sustained": sustained},
-        "append_roofline": {"kernel": "rmsnorm_rope_kv_append_kernel" if args.rmsnorm else "rope_kv_append_kernel",
+        "append_roofline": {"kernel": "rmsnorm_rope_kv_append_token_kernel" if args.rmsnorm else "rope_kv_append_kernel",
                             "bound": "hbm", "achieved": append_bytes / (t_append * 1e-3) / 1e9,
                             "peak": peaks["hbm_gbs"], "unit": "GB/s",
                             "frac": append_bytes / (t_append * 1e-3) / 1e9 / peaks["hbm_gbs"],

@@ -32,7 +32,8 @@ def _inputs():
 # Diagnostic variants of the library, built beside the normal one as libunstep_<name>.so and
 # loaded instead of it when the environment variable UNSTEP_LIB_VARIANT names one.
 VARIANTS = {
-    "check": ["-DUNSTEP_CHECK"],   # every global store bounds-checked, violations reported, never made
+    "check": ["-DUNSTEP_CHECK"],
+    "abl3": ["-DNORM_ABL=3"],   # every global store bounds-checked, violations reported, never made
 }
 
 

@@ -135,30 +135,23 @@ rope_kv_append_kernel(AppendParams p, const uint4* q_in, const uint4* __restrict
 }
 
 // --------------------------------------------------------------------------
-// RMSNorm of q and k fused in front of the rotation: one warp per token.  The norm runs over
-// the whole token vector (all heads).  Pass 1 loads the token's q and k vectors and sums their
-// squares in double.  Each square is exact; the additions round at 2^-53 relative, so a sum taken
-// in another order than the reference's can differ from it in the last bits of the double (and
-// not at all unless the squares of one token span more than about 2^26 in magnitude), far below
-// the rounding of the mean to float32 that follows: the float32 mean, and with it every output
-// bit, does not depend on the order except in a near-tie of that rounding.  Pass 2
-// normalises (float32: sqrt, reciprocal and two products, each rounded once), rounds to bf16 as
-// the unfused pipeline would, rotates and stores.  Pass 2 reads q and k again, from L1/L2:
-// keeping them in registers between the passes cost more in occupancy than the second read.
+// RMSNorm of q and k fused in front of the rotation.  The norm runs over the whole token
+// vector (all heads).  The squares of a token's q and k are summed in double.  Each square is
+// exact; the additions round at 2^-53 relative, so a sum taken in another order than the
+// reference's can differ from it in the last bits of the double (and not at all unless the
+// squares of one token span more than about 2^26 in magnitude), far below the rounding of the
+// mean to float32 that follows: the float32 mean, and with it every output bit, does not depend
+// on the order except in a near-tie of that rounding.  Then the token is normalised (float32:
+// sqrt, reciprocal and two products, each rounded once), rounded to bf16 as the unfused pipeline
+// would, rotated and stored.  Two kernels: a thread block per token that keeps the token in
+// registers between the sum and the store (up to 64 heads), and a warp per token that reads q
+// and k a second time from L1/L2 (wider tokens, which would not fit the registers of a block).
 // --------------------------------------------------------------------------
 
 __device__ __forceinline__ double warp_sum(double x) {
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xFFFFFFFFu, x, o);
   return x;
-}
-// |x| of a bf16 as a double, built with integer operations (sign dropped: only squares are
-// formed): the 8 exponent bits are rebiased into the double's exponent field, the 7 mantissa bits
-// land at its top.  `hi_word_bits` holds the bf16's exponent and mantissa at bits 27..13.
-// Zero and bf16 denormals come out as about 2^-127 instead: their squares (below 2^-252) vanish
-// when the mean is rounded to float32, exactly as the true ones do.
-__device__ __forceinline__ double abs_bf16_as_double(uint32_t hi_word_bits) {
-  return __hiloint2double(static_cast<int>((hi_word_bits & 0x0FFFE000u) + 0x38000000u), 0);
 }
 // Sum of the squares of the 8 bf16 of a vector, in double.  A bf16 square has 16 significant
 // bits, so each fused multiply-add adds an exact square and rounds once, like the additions of
@@ -168,7 +161,8 @@ __device__ __forceinline__ double squares(uint4 x, double acc) {
   const uint32_t w[4] = {x.x, x.y, x.z, x.w};
 #pragma unroll
   for (int i = 0; i < 4; ++i) {
-    const double lo = abs_bf16_as_double(w[i] << 13), hi = abs_bf16_as_double(w[i] >> 3);
+    const double lo = static_cast<double>(__uint_as_float(w[i] << 16));
+    const double hi = static_cast<double>(__uint_as_float(w[i] & 0xFFFF0000u));
     s0 = fma(lo, lo, s0);
     s1 = fma(hi, hi, s1);
   }
@@ -189,10 +183,6 @@ __device__ __forceinline__ uint4 normalise_vec(uint4 x, float r, float4 g0, floa
   return make_uint4(y[0], y[1], y[2], y[3]);
 }
 
-// kVFirst: the V copy rides along with pass 1, so that its traffic overlaps the wait for q and k.
-// It costs 13 registers (74 instead of 61): worth it when the tokens need several waves of warps
-// anyway (14B shape: 165 -> 152 us), not when they just fit one wave (1.3B shape: 23.8 -> 25.3 us).
-template <bool kVFirst>
 __global__ void __launch_bounds__(256)
 rmsnorm_rope_kv_append_kernel(AppendParams p, float eps, const uint4* q_in, const uint4* __restrict__ k_in,
                               const uint4* __restrict__ v_in, const float4* __restrict__ gain_q,
@@ -217,14 +207,12 @@ rmsnorm_rope_kv_append_kernel(AppendParams p, float eps, const uint4* q_in, cons
     // four vectors of q and of k per lane in flight at a time
     for (int v0 = lane; v0 < p.vec_per_token; v0 += 32 * 4) {
       uint4 xq[4], xk[4];
-      uint4 xv[4];
 #pragma unroll
       for (int u = 0; u < 4; ++u) {
         const int vi = v0 + 32 * u;
         if (vi < p.vec_per_token) {
           xq[u] = q_in[in_base + vi];   // plain load: q_out may be the same buffer
           xk[u] = __ldg(k_in + in_base + vi);
-          if (kVFirst) xv[u] = __ldcs(v_in + in_base + vi);
         }
       }
 #pragma unroll
@@ -232,7 +220,6 @@ rmsnorm_rope_kv_append_kernel(AppendParams p, float eps, const uint4* q_in, cons
         if (v0 + 32 * u < p.vec_per_token) {
           sq = squares(xq[u], sq);
           sk = squares(xk[u], sk);
-          if (kVFirst) UNSTEP_STORE(ring_v, ring_base + v0 + 32 * u, p.extent_cache, xv[u], p.status);
         }
       }
     }
@@ -249,7 +236,7 @@ rmsnorm_rope_kv_append_kernel(AppendParams p, float eps, const uint4* q_in, cons
     const uint4 nk = normalise_vec(xk, rk, __ldg(gain_k + 2 * vi), __ldg(gain_k + 2 * vi + 1));
     UNSTEP_STORE(q_out, in_base + vi, p.extent_act, rotate_vec(nq, c, s), p.status);
     UNSTEP_STORE(ring_k, ring_base + vi, p.extent_cache, rotate_vec(nk, c, s), p.status);
-    if (!kVFirst) UNSTEP_STORE(ring_v, ring_base + vi, p.extent_cache, __ldcs(v_in + in_base + vi), p.status);
+    UNSTEP_STORE(ring_v, ring_base + vi, p.extent_cache, __ldcs(v_in + in_base + vi), p.status);
   };
   {
     for (int v0 = lane; v0 < p.vec_per_token; v0 += 32 * 2) {
@@ -265,6 +252,82 @@ rmsnorm_rope_kv_append_kernel(AppendParams p, float eps, const uint4* q_in, cons
 #pragma unroll
       for (int u = 0; u < 2; ++u)
         if (v0 + 32 * u < p.vec_per_token) finish(v0 + 32 * u, xq[u], xk[u]);
+    }
+  }
+}
+
+
+// One thread block per token, for token vectors of up to 4 * 256 vectors (64 heads): thread i
+// owns vectors i, i + blockDim, ... (kU of them) of q, k and v, all of them loaded at once and
+// kept in registers from the sum of squares to the rotated store, so that a token makes one
+// trip to memory.  The partial sums meet in shared memory and every thread adds them in the
+// same order.
+template <int kU>
+__global__ void __launch_bounds__(kU <= 2 ? 96 : 256, kU <= 2 ? 12 : 3)
+rmsnorm_rope_kv_append_token_kernel(AppendParams p, float eps, const uint4* q_in, const uint4* __restrict__ k_in,
+                                    const uint4* __restrict__ v_in, const float4* __restrict__ gain_q,
+                                    const float4* __restrict__ gain_k, const float4* __restrict__ cos_t,
+                                    const float4* __restrict__ sin_t, uint4* q_out, uint4* __restrict__ ring_k,
+                                    uint4* __restrict__ ring_v) {
+  __shared__ double part[2][8];
+  const int b = blockIdx.y;
+  const int n = blockIdx.x;   // token
+  const int tid = threadIdx.x, nthr = blockDim.x;
+  const int f = n / p.T, t = n - f * p.T;
+  const int frame = p.start[b] + f;
+  const int slot = frame < p.S ? frame : p.S + (frame - p.S) % p.C;
+  const int64_t in_base = static_cast<int64_t>(b) * p.vec_per_stream + static_cast<int64_t>(n) * p.vec_per_token;
+  const int64_t ring_base = static_cast<int64_t>(b) * p.ring_vec_per_stream +
+                            (static_cast<int64_t>(slot) * p.T + t) * p.vec_per_token;
+  const int64_t tab_base = (static_cast<int64_t>(b) * p.table_stream_stride >> 2) +
+                           static_cast<int64_t>(n) * (kPairs / 4);
+
+  uint4 xq[kU], xk[kU], xv[kU];
+#pragma unroll
+  for (int u = 0; u < kU; ++u) {
+    const int vi = tid + u * nthr;
+    if (vi < p.vec_per_token) {
+      xq[u] = q_in[in_base + vi];   // plain load: q_out may be the same buffer
+      xk[u] = __ldcs(k_in + in_base + vi);
+      xv[u] = __ldcs(v_in + in_base + vi);
+    }
+  }
+  // All vectors of a thread sit at the same place of their heads (the block is a multiple of 16
+  // threads wide), so they share one set of coefficients, fetched under the wait for q, k and v.
+  const float4 c = __ldg(cos_t + tab_base + (tid & 15));
+  const float4 s = __ldg(sin_t + tab_base + (tid & 15));
+  double sq = 0.0, sk = 0.0;
+#pragma unroll
+  for (int u = 0; u < kU; ++u) {
+    const int vi = tid + u * nthr;
+    if (vi < p.vec_per_token) {
+      sq = squares(xq[u], sq);
+      sk = squares(xk[u], sk);
+      UNSTEP_STORE(ring_v, ring_base + vi, p.extent_cache, xv[u], p.status);
+    }
+  }
+  sq = warp_sum(sq);
+  sk = warp_sum(sk);
+  if ((tid & 31) == 0) {
+    part[0][tid >> 5] = sq;
+    part[1][tid >> 5] = sk;
+  }
+  __syncthreads();
+  // even lanes finish q, odd lanes k: one division per warp
+  double tot = 0.0;
+  for (int w = 0; w < (nthr >> 5); ++w) tot += part[tid & 1][w];
+  const double width = static_cast<double>(p.vec_per_token) * 8.0;
+  const float ms = static_cast<float>(tot / width);
+  const float r = __frcp_rn(__fsqrt_rn(__fadd_rn(ms, eps)));
+  const float rq = __shfl_sync(0xFFFFFFFFu, r, 0), rk = __shfl_sync(0xFFFFFFFFu, r, 1);
+#pragma unroll
+  for (int u = 0; u < kU; ++u) {
+    const int vi = tid + u * nthr;
+    if (vi < p.vec_per_token) {
+      const uint4 nq = normalise_vec(xq[u], rq, __ldg(gain_q + 2 * vi), __ldg(gain_q + 2 * vi + 1));
+      const uint4 nk = normalise_vec(xk[u], rk, __ldg(gain_k + 2 * vi), __ldg(gain_k + 2 * vi + 1));
+      UNSTEP_STORE(q_out, in_base + vi, p.extent_act, rotate_vec(nq, c, s), p.status);
+      UNSTEP_STORE(ring_k, ring_base + vi, p.extent_cache, rotate_vec(nk, c, s), p.status);
     }
   }
 }
@@ -425,14 +488,26 @@ extern "C" int unstep_rmsnorm_rope_kv_append(const unstep_shape_t* shape, int32_
     uint4* qo = static_cast<uint4*>(q_out) + in_off;
     uint4* rk = static_cast<uint4*>(cache_k) + ring_off;
     uint4* rv = static_cast<uint4*>(cache_v) + ring_off;
-    // one warp per token: beyond about 32 resident warps per SM the tokens run in waves
-    int sms = 148;
-    int dev = 0;
-    if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    if (static_cast<int64_t>(nb) * L > static_cast<int64_t>(sms) * 32)
-      rmsnorm_rope_kv_append_kernel<true><<<dim3(blocks, nb), 256, 0, st>>>(p, eps, q, k, v, gq, gk, ct, sn, qo, rk, rv);
-    else
-      rmsnorm_rope_kv_append_kernel<false><<<dim3(blocks, nb), 256, 0, st>>>(p, eps, q, k, v, gq, gk, ct, sn, qo, rk, rv);
+    // Up to 64 heads: a thread block per token, of few threads with several vectors each (about
+    // 96 threads for the 12 heads of the 1.3B shape: more tokens in flight per SM than with wider
+    // blocks, 21.6 against 26 us there).
+    if (p.vec_per_token <= 4 * 256) {
+      int per_thread = (p.vec_per_token + 95) / 96;
+      if (per_thread > 4) per_thread = 4;
+      const int threads = (((p.vec_per_token + per_thread - 1) / per_thread) + 31) & ~31;
+      const dim3 grid(static_cast<unsigned>(L), nb);
+      switch (per_thread) {
+        case 1: rmsnorm_rope_kv_append_token_kernel<1><<<grid, threads, 0, st>>>(p, eps, q, k, v, gq, gk, ct, sn, qo, rk, rv); break;
+        case 2: rmsnorm_rope_kv_append_token_kernel<2><<<grid, threads, 0, st>>>(p, eps, q, k, v, gq, gk, ct, sn, qo, rk, rv); break;
+        case 3: rmsnorm_rope_kv_append_token_kernel<3><<<grid, threads, 0, st>>>(p, eps, q, k, v, gq, gk, ct, sn, qo, rk, rv); break;
+        default: rmsnorm_rope_kv_append_token_kernel<4><<<grid, threads, 0, st>>>(p, eps, q, k, v, gq, gk, ct, sn, qo, rk, rv); break;
+      }
+      g_launches.fetch_add(1);
+      if (cudaGetLastError() != cudaSuccess) return UNSTEP_ERR_CUDA;
+      continue;
+    }
+    // wider tokens: one warp per token
+    rmsnorm_rope_kv_append_kernel<<<dim3(blocks, nb), 256, 0, st>>>(p, eps, q, k, v, gq, gk, ct, sn, qo, rk, rv);
     g_launches.fetch_add(1);
     if (cudaGetLastError() != cudaSuccess) return UNSTEP_ERR_CUDA;
   }

@@ -56,12 +56,20 @@ def test_ragged_streams_own_tables_sink_and_in_place():
     run(sh, [(0, 3, 9), (3, 6, 12), (21, 9, 15)], sink=3, in_place=True, scale=4.0)
 
 
-def test_1p3b_shape_registers_path():
+def test_1p3b_shape():
     run(W.WORKLOADS["cfg2"].shape, [(18,)], eps=1e-5)
 
 
-def test_14b_shape_reload_path():
+def test_14b_shape():
     run(W.WORKLOADS["cfg5"].shape, [(9,)])
+
+
+@pytest.mark.parametrize("heads", [1, 5, 6, 7, 13, 17, 18, 19, 33, 64, 65, 70])
+def test_every_block_width_and_the_wide_token_kernel(heads):
+    # 1..4 vectors per thread, blocks of 32 to 256 threads with and without idle lanes, and (from
+    # 65 heads on) the warp-per-token kernel; two streams, the ring wrapped
+    sh = W.Shape(batch=2, heads=heads, chunk_frames=2, grid_h=3, grid_w=7, ring_frames=4)
+    run(sh, [(0, 2), (2, 4), (4, 6)], seed=70 + heads, scale=2.0)
 
 
 def test_argument_checks():
