@@ -75,6 +75,7 @@ class ClockSampler(threading.Thread):
         self.t, self.mhz, self.power, self.mask = [], [], [], []
         self.max_mhz = None
         self._halt = threading.Event()
+        self.ready = threading.Event()     # set after the first sample (NVML start-up can take a while)
         self.error = None
         self.names = {}
 
@@ -99,10 +100,12 @@ class ClockSampler(threading.Thread):
                     watts = nv.nvmlDeviceGetPowerUsage(h) / 1000.0
                 self.power.append(watts)
                 self.mask.append(int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(h)))
+                self.ready.set()
                 n += 1
                 time.sleep(self.period)
         except Exception as exc:  # NVML missing: report it, never fail the benchmark
             self.error = repr(exc)
+            self.ready.set()
 
     def stop(self):
         self._halt.set()
@@ -399,6 +402,7 @@ def run_ours(args):
     sampler = ClockSampler(physical_gpu_index(local_rank)) if rank == 0 else None
     if sampler:
         sampler.start()
+        sampler.ready.wait(timeout=10.0)   # the short first leg must not be over before NVML is up
 
     def timed_leg(n_steps):
         """n_steps back-to-back steps with per-kernel events; returns (total ms, per-kernel arrays,
